@@ -1,0 +1,235 @@
+"""CPU oracle of the batched draft-verification pass. TEST INFRASTRUCTURE ONLY.
+
+Nothing in the product path may import this file: it exists so that tests, the
+smoke check and the benchmark's CPU-baseline leg can compare the CUDA kernels
+with a slow, plain statement of what the paper defines. It shares no code with
+the CUDA path and never imports it.
+
+What it states (paper Section 4.2, "Draft Verification" and "Cascaded Decision
+Rule"; Algorithm 1, Stage 2): the verifier model reads the cached reasoning
+context followed by the step's new tokens (draft step, target step, prompt
+suffix), emits one decision token, and the confidence p_D is the softmax
+probability of that decision token (Eqs. 2-3); the draft's decision is trusted
+when p_D >= gamma and escalated to the target model otherwise (Eq. 4).
+
+The model itself is not defined by the paper beyond its family (decoder-only,
+RMSNorm, rotary positions, grouped-query attention, SwiGLU MLP); those blocks
+are written here from their textbook definitions. All arithmetic is float64 on
+the exactly widened bf16 weights and bf16 context K/V. No tiling, no online
+softmax, no split reductions: each function is the definition written out,
+with numpy matmul as the only library step.
+
+Parity pins (tests/test_oracle_*.py): closed forms for each block, brute-force
+attention with scalar loops, cache-extend == full causal recompute, rotary
+shift invariance, GQA == MHA with repeated heads, softmax sums to one, gate
+end points of Table 3 (gamma = 0 never escalates, gamma > 1 always does),
+batch-permutation equivariance, and the whole forward against the
+`transformers` Qwen2 architecture used as a black-box library routine.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+
+# ----------------------------------------------------------------------------------------------
+# storage formats
+# ----------------------------------------------------------------------------------------------
+
+def widen_bf16(bits: np.ndarray) -> np.ndarray:
+    """uint16 bf16 bit patterns -> float64, exactly (bf16 is the upper half of an fp32)."""
+    u = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return u.view(np.float32).astype(np.float64)
+
+
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """float64 -> nearest bf16 value (ties to even, via fp32), returned as float64. Used only where the
+    cache format is bf16: the K/V a prefill writes are stored rounded."""
+    u = np.ascontiguousarray(x, dtype=np.float64).astype(np.float32).view(np.uint32)
+    r = u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))
+    r &= np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(np.float64)
+
+
+# ----------------------------------------------------------------------------------------------
+# model blocks (textbook definitions)
+# ----------------------------------------------------------------------------------------------
+
+def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) * gain, row-wise."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * gain
+
+
+def rope(y: np.ndarray, positions: np.ndarray, theta: float) -> np.ndarray:
+    """Rotary position embedding, "rotate-half" pairing. y: [n, heads, hd]; positions: [n].
+    Pair (j, j + hd/2) is rotated by the angle pos * theta^(-2j/hd)."""
+    n, _, hd = y.shape
+    half = hd // 2
+    inv_freq = theta ** (-2.0 * np.arange(half, dtype=np.float64) / hd)
+    ang = positions.astype(np.float64)[:, None] * inv_freq[None, :]          # [n, half]
+    c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    a, b = y[..., :half], y[..., half:]
+    return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
+
+
+def silu(z: np.ndarray) -> np.ndarray:
+    return z / (1.0 + np.exp(-z))
+
+
+def attention_extend(q: np.ndarray, k_ctx: np.ndarray, v_ctx: np.ndarray,
+                     k_new: np.ndarray, v_new: np.ndarray) -> np.ndarray:
+    """Grouped-query attention of n new positions over c cached positions (all visible) and over the
+    new positions themselves (causal). q: [n, Hq, hd]; k_ctx, v_ctx: [c, Hkv, hd]; k_new, v_new:
+    [n, Hkv, hd]. Query head h reads kv head h // (Hq // Hkv). Returns [n, Hq, hd]."""
+    n, hq, hd = q.shape
+    c = k_ctx.shape[0]
+    group = hq // k_new.shape[1]
+    keys = np.concatenate([k_ctx, k_new], axis=0)        # [c + n, Hkv, hd]
+    vals = np.concatenate([v_ctx, v_new], axis=0)
+    # new position p (absolute index c + p) may see absolute key indices 0 .. c + p
+    visible = np.arange(c + n)[None, :] <= (c + np.arange(n))[:, None]
+    out = np.empty_like(q)
+    for h in range(hq):
+        kh = h // group
+        s = (q[:, h, :] @ keys[:, kh, :].T) / np.sqrt(float(hd))           # [n, c + n]
+        s = np.where(visible, s, -np.inf)
+        s = s - np.max(s, axis=-1, keepdims=True)
+        p = np.exp(s)
+        p = p / np.sum(p, axis=-1, keepdims=True)
+        out[:, h, :] = p @ vals[:, kh, :]
+    return out
+
+
+class LayerWeights:
+    """One decoder layer's matrices widened to float64 ([out_features, in_features])."""
+
+    def __init__(self, layer: dict):
+        for name in ("wq", "wk", "wv", "wo", "wg", "wu", "wd"):
+            setattr(self, name, widen_bf16(layer[name]))
+        self.norm1 = np.asarray(layer["norm1"], dtype=np.float64)
+        self.norm2 = np.asarray(layer["norm2"], dtype=np.float64)
+
+
+def decoder_layer_extend(x: np.ndarray, lw: LayerWeights, shape, ctx_len: int,
+                         k_ctx: np.ndarray, v_ctx: np.ndarray
+                         ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """One pre-norm decoder layer over the n new positions of one step whose cached context has ctx_len
+    positions. x: [n, d]. Returns (x_out, k_new, v_new) with k_new rotated, both [n, Hkv, hd]."""
+    n = x.shape[0]
+    hq, hkv, hd = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    pos = ctx_len + np.arange(n)
+    a = rmsnorm(x, lw.norm1, shape.rms_eps)
+    q = (a @ lw.wq.T).reshape(n, hq, hd)
+    k = (a @ lw.wk.T).reshape(n, hkv, hd)
+    v = (a @ lw.wv.T).reshape(n, hkv, hd)
+    q = rope(q, pos, shape.rope_theta)
+    k = rope(k, pos, shape.rope_theta)
+    o = attention_extend(q, k_ctx, v_ctx, k, v).reshape(n, hq * hd)
+    x = x + o @ lw.wo.T
+    b = rmsnorm(x, lw.norm2, shape.rms_eps)
+    x = x + (silu(b @ lw.wg.T) * (b @ lw.wu.T)) @ lw.wd.T
+    return x, k, v
+
+
+# ----------------------------------------------------------------------------------------------
+# confidence and gate (paper Eqs. 2-4)
+# ----------------------------------------------------------------------------------------------
+
+def logsumexp_full_vocab(logits: np.ndarray) -> np.ndarray:
+    """log sum_v exp(z_v) over the whole vocabulary (last axis), shifted by the row maximum."""
+    m = np.max(logits, axis=-1, keepdims=True)
+    return (m + np.log(np.sum(np.exp(logits - m), axis=-1, keepdims=True)))[..., 0]
+
+
+def log_softmax_full_vocab(logits: np.ndarray) -> np.ndarray:
+    """log of the softmax over the whole vocabulary (last axis)."""
+    return logits - logsumexp_full_vocab(logits)[..., None]
+
+
+def verdict_confidence(logits: np.ndarray, verdict_ids: Sequence[int]
+                       ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Decision r_D and confidence p_D of Eqs. 2-3. The decision is the verdict token (one of
+    `verdict_ids`) with the largest probability under the full-vocabulary softmax and p_D is that
+    probability; ties go to the earliest entry of `verdict_ids`. logits: [B, V].
+    Returns (conf [B] float64, verdict index [B] int32, log-sum-exp [B] float64)."""
+    lse = logsumexp_full_vocab(logits)
+    pv = np.exp(logits[:, list(verdict_ids)] - lse[:, None])   # [B, n_verdict]
+    verdict = np.argmax(pv, axis=-1).astype(np.int32)   # first maximum
+    conf = pv[np.arange(pv.shape[0]), verdict]
+    return conf, verdict, lse
+
+
+def gate(conf: np.ndarray, tau: float) -> np.ndarray:
+    """Cascade rule of Eq. 4: 1 where the draft verifier's decision is trusted (p_D >= gamma), 0 where
+    the step is escalated to the target model. The comparison is taken in fp32, the precision in which
+    the confidence is stored; a NaN confidence escalates."""
+    c32 = np.asarray(conf, dtype=np.float64).astype(np.float32)
+    return (c32 >= np.float32(tau)).astype(np.uint8)
+
+
+def escalate_list(conf: np.ndarray, tau: float) -> Tuple[np.ndarray, np.ndarray, int]:
+    """Re-gate stored confidences and list the escalated steps in ascending order.
+    Returns (accept mask uint8 [B], escalated step indices int32 [count], count)."""
+    acc = gate(conf, tau)
+    idx = np.nonzero(acc == 0)[0].astype(np.int32)
+    return acc, idx, int(idx.shape[0])
+
+
+# ----------------------------------------------------------------------------------------------
+# whole pass
+# ----------------------------------------------------------------------------------------------
+
+def forward_extend(weights: dict, tokens_per_step: List[np.ndarray], ctx_lens: Sequence[int],
+                   ctx_kv_fn, collect_new_kv: bool = False):
+    """Run every step's new tokens through all layers on top of its cached context.
+
+    ctx_kv_fn(step, layer) -> (K, V) float64 arrays [c_i, Hkv, hd] (K already rotated).
+    Steps never interact (the paper verifies candidates independently, Section 4.3); the layer loop is
+    outermost only so that each layer's weights are widened once.
+    Returns (hidden states per step [n_i, d] before the final norm, optional per-step per-layer new K/V).
+    """
+    shape = weights["shape"]
+    emb = weights["embed"]
+    xs = [widen_bf16(emb[np.asarray(t, dtype=np.int64)]) for t in tokens_per_step]
+    new_kv = [[None] * shape.n_layers for _ in xs] if collect_new_kv else None
+    for li in range(shape.n_layers):
+        lw = LayerWeights(weights["layers"][li])
+        for i in range(len(xs)):
+            k_ctx, v_ctx = ctx_kv_fn(i, li)
+            xs[i], k, v = decoder_layer_extend(xs[i], lw, shape, int(ctx_lens[i]), k_ctx, v_ctx)
+            if collect_new_kv:
+                new_kv[i][li] = (k, v)
+    return xs, new_kv
+
+
+def last_position_logits(weights: dict, xs: List[np.ndarray]) -> np.ndarray:
+    """Final RMSNorm of each step's last new position, then the LM head. Returns [B, V] float64."""
+    shape = weights["shape"]
+    g = np.asarray(weights["final_norm"], dtype=np.float64)
+    h = np.stack([rmsnorm(x[-1:, :], g, shape.rms_eps)[0] for x in xs], axis=0)
+    return h @ widen_bf16(weights["lm_head"]).T
+
+
+def prefill_context(weights: dict, ctx_tokens: List[np.ndarray], store_bf16: bool):
+    """Build each sequence's context K/V by running its context tokens through the model from an empty
+    cache. Returns kv[i][layer] = (K, V), each [c_i, Hkv, hd] float64; rounded to bf16 values when
+    `store_bf16` (the cache format), exact otherwise."""
+    shape = weights["shape"]
+    empty = np.zeros((0, shape.n_kv_heads, shape.head_dim))
+    _, kv = forward_extend(weights, ctx_tokens, [0] * len(ctx_tokens),
+                           lambda i, l: (empty, empty), collect_new_kv=True)
+    if store_bf16:
+        kv = [[(round_to_bf16(k), round_to_bf16(v)) for (k, v) in per_layer] for per_layer in kv]
+    return kv
+
+
+def verify_steps(weights: dict, tokens_per_step: List[np.ndarray], ctx_lens: Sequence[int],
+                 ctx_kv_fn, verdict_ids: Sequence[int], tau: float) -> dict:
+    """The whole verification pass for a batch of steps (Algorithm 1, Stage 2, draft tier).
+    Returns logits [B, V], conf [B], verdict [B], lse [B], accept [B] (1 = trusted, 0 = escalate)."""
+    xs, _ = forward_extend(weights, tokens_per_step, ctx_lens, ctx_kv_fn)
+    logits = last_position_logits(weights, xs)
+    conf, verdict, lse = verdict_confidence(logits, verdict_ids)
+    return {"logits": logits, "conf": conf, "verdict": verdict, "lse": lse, "accept": gate(conf, tau)}

@@ -1,0 +1,60 @@
+"""Host-side checks of the seeded input generators and of the golden gate cases."""
+import os
+
+import numpy as np
+
+from oracle import confspec_oracle as O
+from workloads import CONFIGS, context_kv, get_config, make_batch, model_weights, page_assignment, scaled_config
+
+
+def test_gate_golden_cases():
+    path = os.path.join(os.path.dirname(__file__), "golden", "gate_cases.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(rows) >= 10
+    for conf, tau, want in rows:
+        assert O.gate(np.array([float(conf)]), float(tau)).tolist() == [int(want)], (conf, tau)
+
+
+def test_batches_follow_the_config_recipes():
+    for name, cfg in CONFIGS.items():
+        b = make_batch(cfg)
+        assert b.n_steps == cfg.batch and b.cu_new[-1] == b.step_lens.sum() == b.step_tokens.shape[0]
+        body = b.step_lens - cfg.suffix_len
+        if cfg.step_dist[0] == "uniform":
+            assert body.min() >= cfg.step_dist[1] and body.max() <= cfg.step_dist[2]
+        if cfg.ctx_dist[0] == "uniform":
+            assert b.ctx_lens.min() >= cfg.ctx_dist[1] and b.ctx_lens.max() <= cfg.ctx_dist[2]
+        if cfg.ctx_dist[0] == "lognormal":
+            assert b.ctx_lens.min() >= cfg.ctx_dist[3] and b.ctx_lens.max() <= cfg.ctx_dist[4]
+        assert b.step_tokens.min() >= 3 and b.step_tokens.max() < cfg.model.vocab
+        for i in range(b.n_steps):   # every step ends with the shared verify suffix
+            assert np.array_equal(b.step_tokens[b.cu_new[i + 1] - cfg.suffix_len:b.cu_new[i + 1]], b.suffix)
+        b2 = make_batch(cfg)
+        assert np.array_equal(b.step_tokens, b2.step_tokens) and np.array_equal(b.ctx_lens, b2.ctx_lens)
+
+
+def test_weights_are_seeded_bf16_normals():
+    cfg = get_config("cfg1_tiny")
+    w1, w2 = model_weights(cfg.model, 5, threads=1), model_weights(cfg.model, 5, threads=4)
+    assert np.array_equal(w1["layers"][1]["wd"], w2["layers"][1]["wd"])
+    assert np.array_equal(w1["lm_head"], w2["lm_head"])
+    assert not np.array_equal(w1["lm_head"], w1["embed"])           # untied
+    x = O.widen_bf16(w1["lm_head"])
+    assert abs(x.std() - 0.02) < 5e-4 and abs(x.mean()) < 2e-4
+    assert w1["layers"][0]["wq"].shape == (256, 256) and w1["layers"][0]["wg"].shape == (688, 256)
+    assert np.all(w1["final_norm"] == 1.0)
+
+
+def test_context_kv_and_pages():
+    cfg = scaled_config("cfg2_1p5b_b16", n_layers=2, batch=3)
+    b = make_batch(cfg)
+    k, v = context_kv(cfg, 1, 0, int(b.ctx_lens[1]))
+    assert k.shape == (b.ctx_lens[1], 2, 128) and k.dtype == np.uint16
+    k2, _ = context_kv(cfg, 1, 0, int(b.ctx_lens[1]))
+    assert np.array_equal(k, k2)
+    assert abs(O.widen_bf16(k).std() - cfg.kv_std) < 0.01
+    total, pages = page_assignment(cfg, b.ctx_lens)
+    allp = np.concatenate(pages)
+    assert len(set(allp.tolist())) == allp.shape[0] and allp.max() < total
+    assert [len(p) for p in pages] == [(int(c) + 15) // 16 for c in b.ctx_lens]
+    assert not np.array_equal(pages[0], np.sort(pages[0]))          # scattered, not contiguous

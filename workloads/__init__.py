@@ -1,0 +1,23 @@
+"""Seeded synthetic inputs for the batched verification pass.
+
+This package only *draws* inputs (model tensors, token ids, context K/V, page
+assignments). It contains none of the method's arithmetic: no norm, no
+attention, no softmax, no gate. Both the CPU oracle's tests and the CUDA
+path's tests/bench feed from here so that they see identical bits.
+"""
+from .configs import ModelShape, VerifyConfig, CONFIGS, get_config, scaled_config
+from .generate import (
+    bf16_bits_from_f32,
+    model_weights,
+    plant_verdict_rows,
+    make_batch,
+    context_kv,
+    page_assignment,
+    Batch,
+)
+
+__all__ = [
+    "ModelShape", "VerifyConfig", "CONFIGS", "get_config", "scaled_config",
+    "bf16_bits_from_f32", "model_weights", "plant_verdict_rows", "make_batch",
+    "context_kv", "page_assignment", "Batch",
+]
