@@ -1,0 +1,209 @@
+/*
+ * confspec.h — C ABI of the batched draft-verification pass of confidence-gated cascaded verification.
+ *
+ * What the library computes (paper Section 4.2; Algorithm 1, Stage 2): a batch of candidate reasoning
+ * steps, each appended to its cached reasoning context, is run through one extend-prefill of a
+ * decoder-only transformer; the hidden state of each step's last new position goes through the LM head;
+ * the probability of the decision ("verdict") token under the softmax over the whole vocabulary is the
+ * confidence p_D (Eqs. 2-3); the draft verifier's decision is trusted when p_D >= gamma and the step is
+ * escalated to the target model otherwise (Eq. 4). Every step of that path runs in CUDA kernels written
+ * for sm_100a; there is no CPU fallback.
+ *
+ * Conventions
+ *  - Every function returns an int status (CS_OK = 0). Nothing throws, exits or prints.
+ *  - "host" / "device" in a parameter comment says where the pointer must point. Device pointers are
+ *    plain CUDA device addresses on the current device (for instance torch.Tensor.data_ptr()).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Calls that take a
+ *    stream only enqueue work; results are valid once the stream has been synchronised.
+ *  - Handles are not thread-safe: use one handle from one host thread at a time.
+ *  - bf16 values are passed as uint16_t bit patterns.
+ */
+#ifndef CONFSPEC_H
+#define CONFSPEC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  CS_OK = 0,
+  CS_EINVAL = 1,   /* an argument is out of range or NULL; nothing was launched */
+  CS_ENOMEM = 2,   /* a device or host allocation failed */
+  CS_ECUDA = 3,    /* a CUDA runtime / driver call failed; see cs_last_cuda_error */
+  CS_ETIMEOUT = 4, /* a kernel gave up on a bounded wait (reported by cs_last_status) */
+  CS_ESTATE = 5    /* the call does not fit the handle's state (e.g. sequence not set) */
+};
+
+typedef struct cs_model cs_model;
+typedef struct cs_kv cs_kv;
+
+/* Geometry of the decoder. n_q_heads must be a multiple of n_kv_heads; head_dim is 64 or 128;
+ * d_model, n_q_heads*head_dim and d_ffn must be multiples of 8 (16-byte rows for TMA). */
+typedef struct cs_model_desc {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rope_theta; /* rotary base; pair (j, j + head_dim/2) turns by pos * theta^(-2j/head_dim) */
+  float rms_eps;    /* added to the mean square inside every RMSNorm */
+} cs_model_desc;
+
+/* Weights handed to cs_model_load. Matrices are bf16, row-major [out_features, in_features].
+ * The per-layer members are arrays of n_layers pointers. No biases; embedding and LM head are separate. */
+typedef struct cs_model_tensors {
+  const uint16_t* embed;        /* [vocab, d_model] */
+  const uint16_t* lm_head;      /* [vocab, d_model] */
+  const float* final_norm;      /* [d_model] RMSNorm gain before the LM head */
+  const uint16_t* const* wq;    /* [n_q_heads*head_dim, d_model] */
+  const uint16_t* const* wk;    /* [n_kv_heads*head_dim, d_model] */
+  const uint16_t* const* wv;    /* [n_kv_heads*head_dim, d_model] */
+  const uint16_t* const* wo;    /* [d_model, n_q_heads*head_dim] */
+  const uint16_t* const* wg;    /* [d_ffn, d_model]  SwiGLU gate */
+  const uint16_t* const* wu;    /* [d_ffn, d_model]  SwiGLU up */
+  const uint16_t* const* wd;    /* [d_model, d_ffn]  SwiGLU down */
+  const float* const* norm1;    /* [d_model] gain of the pre-attention RMSNorm */
+  const float* const* norm2;    /* [d_model] gain of the pre-MLP RMSNorm */
+} cs_model_tensors;
+
+/* Library version as major*10000 + minor*100 + patch. */
+int cs_version(void);
+/* Static English text for a status code. */
+const char* cs_strerror(int status);
+/* Text of the last CUDA error seen by a call on this host thread ("" if none). */
+const char* cs_last_cuda_error(void);
+
+/*
+ * cs_model_load — copy a verifier model (the M_D, or M_T for escalated steps, of Algorithm 1) into
+ * library-owned device memory and prepare everything that does not depend on a batch (fused QKV matrix,
+ * TMA descriptors, rotary frequencies).
+ *   desc               host. Geometry.
+ *   tensors            host struct; the tensor pointers inside are host pointers when
+ *                      tensors_on_device == 0, device pointers otherwise. The caller keeps ownership and
+ *                      may free them once the call returns (the copy is synchronous).
+ *   out                receives the handle; release with cs_model_free.
+ * Errors: CS_EINVAL (NULL, bad geometry), CS_ENOMEM, CS_ECUDA (e.g. not an sm_100 device).
+ */
+int cs_model_load(const cs_model_desc* desc, const cs_model_tensors* tensors, int tensors_on_device,
+                  cs_model** out);
+int cs_model_free(cs_model* model);
+
+/*
+ * cs_reserve — size the per-model activation workspace for batches of up to max_steps steps and
+ * max_tokens new tokens in total. Optional: cs_verify_steps / cs_prefill grow the workspace on demand, but
+ * growing synchronises the device, so latency-sensitive callers reserve once up front.
+ */
+int cs_reserve(cs_model* model, int max_steps, int max_tokens);
+
+/*
+ * cs_kv_alloc — the paged bf16 cache of reasoning contexts ("context" of Algorithm 1, which grows by the
+ * accepted steps and is re-read by every verification).
+ * Pool layout (bf16): [n_layers][2 (K, V)][num_pages][n_kv_heads][page_size][head_dim]; K is stored
+ * already rotated. page_size must be 16. The pool is zero-filled at allocation; slots past a sequence's
+ * length inside its last page must hold finite values (they are masked, not skipped).
+ *   dev_pool           device or NULL. When given, caller-owned memory of cs_kv_pool_bytes() bytes,
+ *                      256-byte aligned, already zeroed; otherwise the library allocates and owns the pool.
+ *   max_seqs, max_pages_per_seq   capacity of the page table.
+ */
+int cs_kv_alloc(const cs_model* model, int num_pages, int page_size, int max_seqs, int max_pages_per_seq,
+                void* dev_pool, cs_kv** out);
+int cs_kv_free(cs_kv* kv);
+/* Bytes of pool that cs_kv_alloc needs for this geometry (0 on bad arguments). */
+uint64_t cs_kv_pool_bytes(const cs_model* model, int num_pages, int page_size);
+
+/*
+ * cs_kv_set_seq — define sequence `seq`: its pages, in order, and its cached length.
+ *   page_ids           host int32[n_pages], each in [0, num_pages). Pages may be shared by several
+ *                      sequences (k candidate steps verified on one context).
+ *   ctx_len            cached tokens, 0 <= ctx_len <= n_pages * page_size.
+ * Host-side only; the table is uploaded by the next call that reads it.
+ */
+int cs_kv_set_seq(cs_kv* kv, int seq, const int32_t* page_ids, int n_pages, int ctx_len);
+
+/*
+ * cs_kv_fill — write given K/V into the pages of sequence `seq` for one layer (synthetic contexts in
+ * tests and benchmarks).
+ *   host_k, host_v     host bf16 [ctx_len, n_kv_heads, head_dim]; K already rotated.
+ * Synchronous on `stream`.
+ */
+int cs_kv_fill(cs_kv* kv, int seq, int layer, const uint16_t* host_k, const uint16_t* host_v, void* stream);
+
+/*
+ * cs_prefill — run tokens through the model and APPEND their K/V to the sequences' pages
+ * (context management of Algorithm 1, Stage 3: accepted steps become context). The sequences must have
+ * enough pages set for ctx_len + lens[i]. On success each sequence's ctx_len grows by lens[i].
+ *   seq_ids, lens      host int32[B];  tokens  host int32[sum lens], concatenated per sequence.
+ */
+int cs_prefill(cs_model* model, cs_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
+               const int32_t* lens, int B, void* stream);
+
+/*
+ * cs_verify_steps — the verification pass itself (M.verify of Algorithm 1, Stage 2; Eqs. 2-4).
+ * For step i, the new tokens step_tokens[cu[i] .. cu[i]+step_lens[i]) (draft step, target step and the
+ * verification prompt, as one opaque span) are placed at positions ctx_len .. ctx_len+step_lens[i]-1 after
+ * the cached context of sequence seq_ids[i]; the last position's logits z give
+ *     conf = max_j exp(z[verdict_ids[j]] - logsumexp_v z[v]),   verdict = first j attaining it,
+ *     accept = (conf >= tau)     (fp32 comparison; NaN never accepts).
+ * The cache is read-only here: K/V of the new tokens live in the model's workspace and are discarded.
+ *   ctx_kv             cache handle whose sequences seq_ids[i] have been set.
+ *   seq_ids            host int32[B]. The same sequence may appear several times.
+ *   step_tokens        int32[sum step_lens]; host when tokens_on_device == 0 (copied on `stream`), else
+ *                      device. Ids must lie in [0, vocab) (host tokens are checked; device tokens are clamped).
+ *   step_lens          host int32[B], each >= 1 (verification suffix included).
+ *   verdict_ids        host int32[n_verdict], 1 <= n_verdict <= 8, ids in [0, vocab).
+ *   tau                threshold gamma of Eq. 4; NaN is rejected with CS_EINVAL.
+ *   out_conf           device float[B].
+ *   out_accept         device uint8[B]: 1 = the draft decision is trusted, 0 = escalate.
+ *   out_verdict        device int32[B] or NULL: index into verdict_ids of the decision r_D.
+ * Asynchronous on `stream`. The residual-stream projections accumulate with floating-point atomics, so
+ * repeated calls agree to rounding, not bit for bit.
+ * Errors: CS_EINVAL before any launch; CS_ESTATE for an unset sequence; CS_ENOMEM / CS_ECUDA.
+ */
+int cs_verify_steps(cs_model* model, const cs_kv* ctx_kv, const int32_t* seq_ids, int B,
+                    const int32_t* step_tokens, int tokens_on_device, const int32_t* step_lens,
+                    const int32_t* verdict_ids, int n_verdict, float tau,
+                    float* out_conf, uint8_t* out_accept, int32_t* out_verdict, void* stream);
+
+/*
+ * cs_escalate_mask — re-apply the rule of Eq. 4 to stored confidences for another threshold and list
+ * the steps that must go to the target model, without leaving the device.
+ *   conf               device float[B].
+ *   out_accept         device uint8[B] or NULL.
+ *   out_escalate_idx   device int32[B]: the first *out_escalate_count entries are the indices of the
+ *                      escalated steps in ascending order; the rest is left untouched.
+ *   out_escalate_count device int32[1].
+ * B <= 65536. Asynchronous on `stream`.
+ */
+int cs_escalate_mask(const float* conf, int B, float tau, uint8_t* out_accept,
+                     int32_t* out_escalate_idx, int32_t* out_escalate_count, void* stream);
+
+/*
+ * Debug / test access. cs_set_keep_logits(model, 1) makes every later cs_verify_steps also write the full
+ * last-position logits (fp32 [B, vocab]) into the workspace; cs_get_last_logits copies them to
+ * dev_out (device float[B*vocab]) on `stream`. cs_get_last_lse copies the per-step logsumexp
+ * (device float[B]). cs_last_status synchronises `stream` and returns CS_ETIMEOUT if any kernel since the
+ * previous query gave up on a bounded wait, else CS_OK.
+ */
+int cs_set_keep_logits(cs_model* model, int keep);
+int cs_get_last_logits(cs_model* model, float* dev_out, int B, void* stream);
+int cs_get_last_lse(cs_model* model, float* dev_out, int B, void* stream);
+int cs_last_status(cs_model* model, void* stream);
+
+/*
+ * Per-stage entry points. They run single kernels of the pass on caller-provided device buffers so that
+ * each can be checked against the oracle's corresponding block, and timed, in isolation.
+ */
+/* out[M,N] (+)= a[M,K] * w[N,K]^T on the tcgen05 tensor cores. a, w bf16 row-major.
+ *   epilogue 0: out bf16 [M,N] = result.
+ *   epilogue 1: out fp32 [M,N] += result (atomic adds; split along K over the SMs).
+ *   epilogue 2: w2 is a second [N,K] matrix; out bf16 [M,N] = silu(a*w^T) * (a*w2^T).
+ * K and N multiples of 8. Asynchronous on `stream`. */
+int cs_gemm_bf16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* out,
+                 int M, int N, int K, int epilogue, void* stream);
+/* out bf16 [rows, d] = RMSNorm(x fp32 [rows, d]; gain fp32 [d], eps). */
+int cs_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps, void* stream);
+/* Number of kernels the library has launched on this host thread since the last call of this function. */
+int64_t cs_take_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CONFSPEC_H */

@@ -119,6 +119,8 @@ def decoder_layer_extend(x: np.ndarray, lw: LayerWeights, shape, ctx_len: int,
     positions. x: [n, d]. Returns (x_out, k_new, v_new) with k_new rotated, both [n, Hkv, hd]."""
     n = x.shape[0]
     hq, hkv, hd = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    if n == 0:  # no new position: nothing to compute, nothing to cache
+        return x, np.zeros((0, hkv, hd)), np.zeros((0, hkv, hd))
     pos = ctx_len + np.arange(n)
     a = rmsnorm(x, lw.norm1, shape.rms_eps)
     q = (a @ lw.wq.T).reshape(n, hq, hd)

@@ -1,0 +1,766 @@
+// C ABI of the library: handles, argument checks, host-side batch metadata and the launch sequence.
+#include "../../include/confspec.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "gemm.h"
+#include "kernels.h"
+
+using namespace cs;
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+int cuda_fail(cudaError_t e, const char* what) {
+  g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+  cudaGetLastError();
+  return e == cudaErrorMemoryAllocation ? CS_ENOMEM : CS_ECUDA;
+}
+#define CS_CUDA(call)                                     \
+  do {                                                    \
+    cudaError_t e__ = (call);                             \
+    if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+  } while (0)
+
+constexpr int kPageSize = 16;
+constexpr int kStagingRing = 4;
+
+struct LayerDev {
+  uint16_t *wqkv, *wo, *wg, *wu, *wd;
+  float *norm1, *norm2;
+  CUtensorMap tm_wqkv, tm_wo, tm_wg, tm_wu, tm_wd;
+};
+
+struct DevBuf {
+  void* p = nullptr;
+  size_t cap = 0;
+  int ensure(size_t bytes) {
+    if (bytes <= cap) return CS_OK;
+    if (p) {
+      cudaDeviceSynchronize();
+      cudaFree(p);
+      p = nullptr;
+      cap = 0;
+    }
+    const size_t want = bytes + bytes / 4 + 256;
+    cudaError_t e = cudaMalloc(&p, want);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(workspace)");
+    cap = want;
+    return CS_OK;
+  }
+  void release() {
+    if (p) cudaFree(p);
+    p = nullptr;
+    cap = 0;
+  }
+};
+
+struct Staging {
+  int32_t* host[kStagingRing] = {nullptr, nullptr, nullptr, nullptr};
+  size_t host_cap[kStagingRing] = {0, 0, 0, 0};
+  cudaEvent_t ev[kStagingRing] = {nullptr, nullptr, nullptr, nullptr};
+  bool pending[kStagingRing] = {false, false, false, false};
+  int next = 0;
+  DevBuf dev;
+};
+
+}  // namespace
+
+struct cs_model {
+  cs_model_desc d;
+  int q_dim, kv_dim, n_qkv;
+  uint16_t *embed = nullptr, *lm_head = nullptr;
+  float* final_norm = nullptr;
+  double* inv_freq = nullptr;
+  std::vector<LayerDev> layers;
+  std::vector<void*> owned;
+  CUtensorMap tm_lm;
+  // workspace
+  DevBuf x, a, qkv, attn_o, hmlp, rope, h_last, lm_part, vlogits, logits, lse, attn_part_o, attn_part_ml;
+  uint32_t* status = nullptr;
+  Staging stg;
+  bool keep_logits = false;
+  int last_B = 0;
+};
+
+struct cs_kv {
+  const cs_model* model;
+  int num_pages, page_size, max_seqs, max_pages_per_seq;
+  uint16_t* pool = nullptr;
+  bool own_pool = false;
+  size_t plane_elems;  // elements of one (layer, K or V) plane
+  CUtensorMap tm_pool;
+  int32_t* table_host = nullptr;  // pinned [max_seqs, max_pages_per_seq]
+  int32_t* table_dev = nullptr;
+  std::vector<int32_t> ctx_len, n_pages;  // per sequence; ctx_len < 0 = not set
+  bool dirty = true;
+  cudaEvent_t upload_ev = nullptr;
+  bool upload_pending = false;
+  DevBuf fill_tmp;
+};
+
+namespace {
+
+int upload_table(cs_kv* kv, cudaStream_t s) {
+  if (!kv->dirty) return CS_OK;
+  CS_CUDA(cudaMemcpyAsync(kv->table_dev, kv->table_host,
+                          sizeof(int32_t) * static_cast<size_t>(kv->max_seqs) * kv->max_pages_per_seq,
+                          cudaMemcpyHostToDevice, s));
+  CS_CUDA(cudaEventRecord(kv->upload_ev, s));
+  kv->upload_pending = true;
+  kv->dirty = false;
+  return CS_OK;
+}
+
+// Host staging slot of at least `ints` int32, safe to overwrite.
+int staging_slot(Staging& st, size_t ints, int* slot_out) {
+  const int slot = st.next;
+  st.next = (st.next + 1) % kStagingRing;
+  if (st.pending[slot]) {
+    CS_CUDA(cudaEventSynchronize(st.ev[slot]));
+    st.pending[slot] = false;
+  }
+  if (!st.ev[slot]) CS_CUDA(cudaEventCreateWithFlags(&st.ev[slot], cudaEventDisableTiming));
+  if (st.host_cap[slot] < ints) {
+    if (st.host[slot]) cudaFreeHost(st.host[slot]);
+    st.host[slot] = nullptr;
+    const size_t want = ints + ints / 2 + 1024;
+    CS_CUDA(cudaMallocHost(reinterpret_cast<void**>(&st.host[slot]), want * sizeof(int32_t)));
+    st.host_cap[slot] = want;
+  }
+  *slot_out = slot;
+  return CS_OK;
+}
+
+struct BatchLayout {
+  int B = 0, T = 0;
+  size_t off_cu, off_ctx, off_seq, off_pos, off_tseq, off_tok, off_items, off_merges, total;
+  int n_items = 0, n_merges = 0, n_slots = 0;
+};
+
+// Splits the attention of every (step, kv head, 64-row query tile) into key-tile ranges of similar length so
+// that the grid is a few times the SM count, longest ranges first.
+void build_attention_work(const cs_model* m, int B, const int32_t* lens, const int32_t* ctx, std::vector<AttnItem>& items,
+                          std::vector<AttnMerge>& merges, int* n_slots) {
+  const int G = m->d.n_q_heads / m->d.n_kv_heads;
+  long total_tiles = 0;
+  for (int i = 0; i < B; ++i) {
+    const int rows = lens[i] * G;
+    const int ctx_tiles = (ctx[i] + 63) / 64;
+    for (int q0 = 0; q0 < rows; q0 += 64) {
+      const int p_max = std::min(lens[i] - 1, (q0 + 63) / G);
+      total_tiles += static_cast<long>(ctx_tiles + p_max / 64 + 1) * m->d.n_kv_heads;
+    }
+  }
+  const long target_items = 3L * kNumSMs;
+  const int chunk = static_cast<int>(std::max<long>(8, (total_tiles + target_items - 1) / target_items));
+  items.clear();
+  merges.clear();
+  int slots = 0;
+  for (int i = 0; i < B; ++i) {
+    const int rows = lens[i] * G;
+    const int ctx_tiles = (ctx[i] + 63) / 64;
+    for (int h = 0; h < m->d.n_kv_heads; ++h) {
+      for (int q0 = 0; q0 < rows; q0 += 64) {
+        const int p_max = std::min(lens[i] - 1, (q0 + 63) / G);
+        const int nt = ctx_tiles + p_max / 64 + 1;
+        int splits = (nt + chunk - 1) / chunk;
+        if (nt < chunk + chunk / 2) splits = 1;
+        if (splits <= 1) {
+          items.push_back(AttnItem{i, h, q0, 0, nt, -1, 0, 0});
+        } else {
+          merges.push_back(AttnMerge{i, h, q0, slots, splits, 0, 0, 0});
+          for (int s = 0; s < splits; ++s) {
+            const int b = static_cast<int>(static_cast<long>(nt) * s / splits);
+            const int e = static_cast<int>(static_cast<long>(nt) * (s + 1) / splits);
+            items.push_back(AttnItem{i, h, q0, b, e, slots++, 0, 0});
+          }
+        }
+      }
+    }
+  }
+  std::stable_sort(items.begin(), items.end(), [](const AttnItem& a, const AttnItem& b) {
+    return (a.tile_end - a.tile_begin) > (b.tile_end - b.tile_begin);
+  });
+  *n_slots = slots;
+}
+
+int check_model_desc(const cs_model_desc* d) {
+  if (!d) return CS_EINVAL;
+  if (d->n_layers < 1 || d->d_model < 8 || d->n_q_heads < 1 || d->n_kv_heads < 1 || d->d_ffn < 8 || d->vocab < 1)
+    return CS_EINVAL;
+  if (d->head_dim != 64 && d->head_dim != 128) return CS_EINVAL;
+  if (d->n_q_heads % d->n_kv_heads) return CS_EINVAL;
+  if (d->d_model % 8 || d->d_ffn % 8) return CS_EINVAL;
+  if (!(d->rope_theta > 0.f) || !(d->rms_eps >= 0.f)) return CS_EINVAL;
+  return CS_OK;
+}
+
+template <typename T>
+int dev_copy(cs_model* m, T** dst, const T* src, size_t n, bool src_dev) {
+  void* p = nullptr;
+  cudaError_t e = cudaMalloc(&p, n * sizeof(T));
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(weights)");
+  m->owned.push_back(p);
+  CS_CUDA(cudaMemcpy(p, src, n * sizeof(T), src_dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice));
+  *dst = static_cast<T*>(p);
+  return CS_OK;
+}
+
+// The forward over all layers for a staged batch. When `append_kv` is given the new K/V of every layer are
+// also written to that cache's pages.
+int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout& L, const int32_t* dev_meta,
+               const int32_t* d_tok, cudaStream_t s) {
+  const cs_model_desc& d = m->d;
+  const int T = L.T;
+  const int32_t* d_cu = dev_meta + L.off_cu;
+  const int32_t* d_ctx = dev_meta + L.off_ctx;
+  const int32_t* d_seq = dev_meta + L.off_seq;
+  const int32_t* d_pos = dev_meta + L.off_pos;
+  const int32_t* d_tseq = dev_meta + L.off_tseq;
+  const AttnItem* d_items = reinterpret_cast<const AttnItem*>(dev_meta + L.off_items);
+  const AttnMerge* d_merges = reinterpret_cast<const AttnMerge*>(dev_meta + L.off_merges);
+
+  float* x = static_cast<float*>(m->x.p);
+  uint16_t* a = static_cast<uint16_t*>(m->a.p);
+  uint16_t* qkv = static_cast<uint16_t*>(m->qkv.p);
+  uint16_t* attn_o = static_cast<uint16_t*>(m->attn_o.p);
+  uint16_t* hmlp = static_cast<uint16_t*>(m->hmlp.p);
+  float2* rope = static_cast<float2*>(m->rope.p);
+
+  CUtensorMap tm_a, tm_o, tm_h, tm_qkv_attn;
+  if (!make_gemm_operand_map(&tm_a, a, T, d.d_model) || !make_gemm_operand_map(&tm_o, attn_o, T, m->q_dim) ||
+      !make_gemm_operand_map(&tm_h, hmlp, T, d.d_ffn) ||
+      !make_tensor_map_bf16(&tm_qkv_attn, qkv, T, m->n_qkv, kPageSize, 64, true)) {
+    g_cuda_error = "cuTensorMapEncodeTiled failed for an activation buffer";
+    return CS_ECUDA;
+  }
+
+  CS_CUDA(launch_embed(d_tok, m->embed, x, T, d.d_model, d.vocab, s));
+  CS_CUDA(launch_rope_table(d_pos, m->inv_freq, rope, T, d.head_dim / 2, s));
+
+  AttnParams ap;
+  ap.qkv = qkv;
+  ap.out = attn_o;
+  ap.cu_new = d_cu;
+  ap.ctx_len = d_ctx;
+  ap.seq_id = d_seq;
+  ap.page_table = kv->table_dev;
+  ap.max_pages_per_seq = kv->max_pages_per_seq;
+  ap.n_q_heads = d.n_q_heads;
+  ap.n_kv_heads = d.n_kv_heads;
+  ap.head_dim = d.head_dim;
+  ap.n_qkv = m->n_qkv;
+  ap.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(d.head_dim)));
+  ap.part_o = static_cast<float*>(m->attn_part_o.p);
+  ap.part_ml = static_cast<float*>(m->attn_part_ml.p);
+  ap.status = m->status;
+  const int plane_rows = kv->num_pages * d.n_kv_heads * kPageSize;
+
+  for (int l = 0; l < d.n_layers; ++l) {
+    const LayerDev& lw = m->layers[l];
+    CS_CUDA(launch_rmsnorm(x, lw.norm1, a, T, d.d_model, d.rms_eps, s));
+    CS_CUDA(gemm_bf16(tm_a, lw.tm_wqkv, nullptr, qkv, T, m->n_qkv, d.d_model, kEpiStoreBf16, m->status, s));
+    CS_CUDA(launch_rope_apply(qkv, rope, T, m->n_qkv, d.n_q_heads + d.n_kv_heads, d.head_dim, s));
+    ap.k_row_base = (2 * l) * plane_rows;
+    ap.v_row_base = (2 * l + 1) * plane_rows;
+    CS_CUDA(launch_attention(ap, kv->tm_pool, tm_qkv_attn, d_items, L.n_items, d_merges, L.n_merges, s));
+    if (append_kv) {
+      CS_CUDA(launch_kv_scatter(qkv + m->q_dim, qkv + m->q_dim + m->kv_dim, m->n_qkv, d_tseq, d_pos, 0, 0,
+                                append_kv->table_dev, append_kv->max_pages_per_seq,
+                                append_kv->pool + static_cast<size_t>(2 * l) * append_kv->plane_elems,
+                                append_kv->pool + static_cast<size_t>(2 * l + 1) * append_kv->plane_elems,
+                                d.n_kv_heads, d.head_dim, kPageSize, T, s));
+    }
+    CS_CUDA(gemm_bf16(tm_o, lw.tm_wo, nullptr, x, T, d.d_model, m->q_dim, kEpiResidAdd, m->status, s));
+    CS_CUDA(launch_rmsnorm(x, lw.norm2, a, T, d.d_model, d.rms_eps, s));
+    CS_CUDA(gemm_bf16(tm_a, lw.tm_wg, &lw.tm_wu, hmlp, T, d.d_ffn, d.d_model, kEpiSwiGLU, m->status, s));
+    CS_CUDA(gemm_bf16(tm_h, lw.tm_wd, nullptr, x, T, d.d_model, d.d_ffn, kEpiResidAdd, m->status, s));
+  }
+  return CS_OK;
+}
+
+int ensure_workspace(cs_model* m, int B, int T) {
+  const cs_model_desc& d = m->d;
+  int rc;
+  const size_t t = static_cast<size_t>(T);
+  if ((rc = m->x.ensure(t * d.d_model * 4))) return rc;
+  if ((rc = m->a.ensure(t * d.d_model * 2))) return rc;
+  if ((rc = m->qkv.ensure(t * m->n_qkv * 2))) return rc;
+  if ((rc = m->attn_o.ensure(t * m->q_dim * 2))) return rc;
+  if ((rc = m->hmlp.ensure(t * d.d_ffn * 2))) return rc;
+  if ((rc = m->rope.ensure(t * (d.head_dim / 2) * sizeof(float2)))) return rc;
+  const size_t bp = static_cast<size_t>((B + 63) / 64) * 64;
+  if ((rc = m->h_last.ensure(bp * d.d_model * 2))) return rc;
+  if ((rc = m->lm_part.ensure(static_cast<size_t>((B + 63) / 64) * 2 * kNumSMs * 64 * 4))) return rc;
+  if ((rc = m->vlogits.ensure(bp * 8 * 4))) return rc;
+  if ((rc = m->lse.ensure(bp * 4))) return rc;
+  if (m->keep_logits && (rc = m->logits.ensure(static_cast<size_t>(B) * d.vocab * 4))) return rc;
+  return CS_OK;
+}
+
+// Checks a batch, writes its metadata into a staging slot and enqueues the upload.
+int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, const int32_t* tokens,
+                int tokens_on_device, const int32_t* lens, BatchLayout* out, const int32_t** dev_meta,
+                const int32_t** dev_tokens, cudaStream_t s) {
+  long T = 0;
+  for (int i = 0; i < B; ++i) {
+    if (lens[i] < 1) return CS_EINVAL;
+    if (seq_ids[i] < 0 || seq_ids[i] >= kv->max_seqs) return CS_EINVAL;
+    if (kv->ctx_len[seq_ids[i]] < 0) return CS_ESTATE;
+    T += lens[i];
+    if (T > (1 << 24)) return CS_EINVAL;
+  }
+  if (!tokens_on_device)
+    for (long t = 0; t < T; ++t)
+      if (tokens[t] < 0 || tokens[t] >= m->d.vocab) return CS_EINVAL;
+
+  std::vector<int32_t> ctx(B);
+  for (int i = 0; i < B; ++i) ctx[i] = kv->ctx_len[seq_ids[i]];
+  std::vector<AttnItem> items;
+  std::vector<AttnMerge> merges;
+  int n_slots = 0;
+  build_attention_work(m, B, lens, ctx.data(), items, merges, &n_slots);
+
+  BatchLayout L;
+  L.B = B;
+  L.T = static_cast<int>(T);
+  size_t o = 0;
+  auto take = [&o](size_t n) { size_t r = o; o += (n + 3) & ~size_t(3); return r; };  // keep 16-byte alignment
+  L.off_cu = take(B + 1);
+  L.off_ctx = take(B);
+  L.off_seq = take(B);
+  L.off_pos = take(T);
+  L.off_tseq = take(T);
+  L.off_tok = take(tokens_on_device ? 0 : T);
+  L.off_items = take(items.size() * 8);
+  L.off_merges = take(merges.size() * 8);
+  L.total = o;
+  L.n_items = static_cast<int>(items.size());
+  L.n_merges = static_cast<int>(merges.size());
+  L.n_slots = n_slots;
+
+  int rc;
+  if ((rc = ensure_workspace(m, B, L.T))) return rc;
+  const int hd = m->d.head_dim;
+  if ((rc = m->attn_part_o.ensure(static_cast<size_t>(std::max(1, n_slots)) * 64 * hd * 4))) return rc;
+  if ((rc = m->attn_part_ml.ensure(static_cast<size_t>(std::max(1, n_slots)) * 64 * 2 * 4))) return rc;
+  if ((rc = m->stg.dev.ensure(L.total * 4))) return rc;
+  int slot;
+  if ((rc = staging_slot(m->stg, L.total, &slot))) return rc;
+  int32_t* h = m->stg.host[slot];
+  int32_t* cu = h + L.off_cu;
+  cu[0] = 0;
+  for (int i = 0; i < B; ++i) {
+    cu[i + 1] = cu[i] + lens[i];
+    h[L.off_ctx + i] = ctx[i];
+    h[L.off_seq + i] = seq_ids[i];
+    for (int p = 0; p < lens[i]; ++p) {
+      h[L.off_pos + cu[i] + p] = ctx[i] + p;
+      h[L.off_tseq + cu[i] + p] = seq_ids[i];
+    }
+  }
+  if (!tokens_on_device) std::memcpy(h + L.off_tok, tokens, sizeof(int32_t) * T);
+  if (!items.empty()) std::memcpy(h + L.off_items, items.data(), items.size() * sizeof(AttnItem));
+  if (!merges.empty()) std::memcpy(h + L.off_merges, merges.data(), merges.size() * sizeof(AttnMerge));
+  CS_CUDA(cudaMemcpyAsync(m->stg.dev.p, h, L.total * 4, cudaMemcpyHostToDevice, s));
+  CS_CUDA(cudaEventRecord(m->stg.ev[slot], s));
+  m->stg.pending[slot] = true;
+  *out = L;
+  *dev_meta = static_cast<const int32_t*>(m->stg.dev.p);
+  *dev_tokens = tokens_on_device ? tokens : *dev_meta + L.off_tok;
+  return CS_OK;
+}
+
+uint32_t* g_test_status = nullptr;
+
+}  // namespace
+
+extern "C" {
+
+int cs_version(void) { return 100; }
+
+const char* cs_strerror(int status) {
+  switch (status) {
+    case CS_OK: return "ok";
+    case CS_EINVAL: return "invalid argument";
+    case CS_ENOMEM: return "out of memory";
+    case CS_ECUDA: return "CUDA error";
+    case CS_ETIMEOUT: return "a kernel gave up on a bounded wait";
+    case CS_ESTATE: return "call does not fit the handle's state";
+    default: return "unknown status";
+  }
+}
+
+const char* cs_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+int64_t cs_take_launch_count(void) { return take_launch_count(); }
+
+int cs_model_load(const cs_model_desc* desc, const cs_model_tensors* t, int on_dev, cs_model** out) {
+  if (!out) return CS_EINVAL;
+  *out = nullptr;
+  int rc = check_model_desc(desc);
+  if (rc) return rc;
+  if (!t || !t->embed || !t->lm_head || !t->final_norm || !t->wq || !t->wk || !t->wv || !t->wo || !t->wg || !t->wu ||
+      !t->wd || !t->norm1 || !t->norm2)
+    return CS_EINVAL;
+  for (int l = 0; l < desc->n_layers; ++l)
+    if (!t->wq[l] || !t->wk[l] || !t->wv[l] || !t->wo[l] || !t->wg[l] || !t->wu[l] || !t->wd[l] || !t->norm1[l] ||
+        !t->norm2[l])
+      return CS_EINVAL;
+  int dev = 0;
+  cudaDeviceProp prop;
+  CS_CUDA(cudaGetDevice(&dev));
+  CS_CUDA(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) {
+    g_cuda_error = "this library contains sm_100a code only; the current device is not compute capability 10.x";
+    return CS_ECUDA;
+  }
+  cs_model* m = new (std::nothrow) cs_model();
+  if (!m) return CS_ENOMEM;
+  m->d = *desc;
+  m->q_dim = desc->n_q_heads * desc->head_dim;
+  m->kv_dim = desc->n_kv_heads * desc->head_dim;
+  m->n_qkv = m->q_dim + 2 * m->kv_dim;
+  const bool sd = on_dev != 0;
+  const size_t dm = desc->d_model, V = desc->vocab, F = desc->d_ffn;
+#define CS_TRY(expr)     \
+  do {                   \
+    rc = (expr);         \
+    if (rc) {            \
+      cs_model_free(m);  \
+      return rc;         \
+    }                    \
+  } while (0)
+  CS_TRY(dev_copy(m, &m->embed, t->embed, V * dm, sd));
+  CS_TRY(dev_copy(m, &m->lm_head, t->lm_head, V * dm, sd));
+  CS_TRY(dev_copy(m, &m->final_norm, t->final_norm, dm, sd));
+  m->layers.resize(desc->n_layers);
+  for (int l = 0; l < desc->n_layers; ++l) {
+    LayerDev& lw = m->layers[l];
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, static_cast<size_t>(m->n_qkv) * dm * 2);
+    if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc(wqkv)"); cs_model_free(m); return rc; }
+    m->owned.push_back(p);
+    lw.wqkv = static_cast<uint16_t*>(p);
+    const cudaMemcpyKind kind = sd ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    e = cudaMemcpy(lw.wqkv, t->wq[l], static_cast<size_t>(m->q_dim) * dm * 2, kind);
+    if (e == cudaSuccess) e = cudaMemcpy(lw.wqkv + static_cast<size_t>(m->q_dim) * dm, t->wk[l], static_cast<size_t>(m->kv_dim) * dm * 2, kind);
+    if (e == cudaSuccess) e = cudaMemcpy(lw.wqkv + static_cast<size_t>(m->q_dim + m->kv_dim) * dm, t->wv[l], static_cast<size_t>(m->kv_dim) * dm * 2, kind);
+    if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy(wqkv)"); cs_model_free(m); return rc; }
+    CS_TRY(dev_copy(m, &lw.wo, t->wo[l], dm * m->q_dim, sd));
+    CS_TRY(dev_copy(m, &lw.wg, t->wg[l], F * dm, sd));
+    CS_TRY(dev_copy(m, &lw.wu, t->wu[l], F * dm, sd));
+    CS_TRY(dev_copy(m, &lw.wd, t->wd[l], dm * F, sd));
+    CS_TRY(dev_copy(m, &lw.norm1, t->norm1[l], dm, sd));
+    CS_TRY(dev_copy(m, &lw.norm2, t->norm2[l], dm, sd));
+    if (!make_gemm_operand_map(&lw.tm_wqkv, lw.wqkv, m->n_qkv, desc->d_model) ||
+        !make_gemm_operand_map(&lw.tm_wo, lw.wo, desc->d_model, m->q_dim) ||
+        !make_gemm_operand_map(&lw.tm_wg, lw.wg, desc->d_ffn, desc->d_model) ||
+        !make_gemm_operand_map(&lw.tm_wu, lw.wu, desc->d_ffn, desc->d_model) ||
+        !make_gemm_operand_map(&lw.tm_wd, lw.wd, desc->d_model, desc->d_ffn)) {
+      g_cuda_error = "cuTensorMapEncodeTiled failed for a weight matrix";
+      cs_model_free(m);
+      return CS_ECUDA;
+    }
+  }
+  if (!make_gemm_operand_map(&m->tm_lm, m->lm_head, desc->vocab, desc->d_model)) {
+    g_cuda_error = "cuTensorMapEncodeTiled failed for the LM head";
+    cs_model_free(m);
+    return CS_ECUDA;
+  }
+  {
+    const int half = desc->head_dim / 2;
+    std::vector<double> f(half);
+    for (int j = 0; j < half; ++j)
+      f[j] = std::pow(static_cast<double>(desc->rope_theta), -2.0 * j / static_cast<double>(desc->head_dim));
+    CS_TRY(dev_copy(m, &m->inv_freq, f.data(), static_cast<size_t>(half), false));
+  }
+  {
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, 256);
+    if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc(status)"); cs_model_free(m); return rc; }
+    m->owned.push_back(p);
+    m->status = static_cast<uint32_t*>(p);
+    cudaMemset(p, 0, 256);
+  }
+#undef CS_TRY
+  CS_CUDA(cudaDeviceSynchronize());
+  *out = m;
+  return CS_OK;
+}
+
+int cs_model_free(cs_model* m) {
+  if (!m) return CS_OK;
+  cudaDeviceSynchronize();
+  for (void* p : m->owned) cudaFree(p);
+  DevBuf* bufs[] = {&m->x, &m->a, &m->qkv, &m->attn_o, &m->hmlp, &m->rope, &m->h_last, &m->lm_part, &m->vlogits,
+                    &m->logits, &m->lse, &m->attn_part_o, &m->attn_part_ml, &m->stg.dev};
+  for (DevBuf* b : bufs) b->release();
+  for (int i = 0; i < kStagingRing; ++i) {
+    if (m->stg.host[i]) cudaFreeHost(m->stg.host[i]);
+    if (m->stg.ev[i]) cudaEventDestroy(m->stg.ev[i]);
+  }
+  delete m;
+  return CS_OK;
+}
+
+int cs_reserve(cs_model* m, int max_steps, int max_tokens) {
+  if (!m || max_steps < 1 || max_tokens < max_steps) return CS_EINVAL;
+  return ensure_workspace(m, max_steps, max_tokens);
+}
+
+uint64_t cs_kv_pool_bytes(const cs_model* m, int num_pages, int page_size) {
+  if (!m || num_pages < 1 || page_size != kPageSize) return 0;
+  return static_cast<uint64_t>(m->d.n_layers) * 2 * num_pages * m->d.n_kv_heads * page_size * m->d.head_dim * 2;
+}
+
+int cs_kv_alloc(const cs_model* m, int num_pages, int page_size, int max_seqs, int max_pages_per_seq, void* dev_pool,
+                cs_kv** out) {
+  if (!out) return CS_EINVAL;
+  *out = nullptr;
+  if (!m || num_pages < 1 || page_size != kPageSize || max_seqs < 1 || max_pages_per_seq < 1) return CS_EINVAL;
+  const uint64_t rows = static_cast<uint64_t>(m->d.n_layers) * 2 * num_pages * m->d.n_kv_heads * page_size;
+  if (rows >= (1ull << 31)) return CS_EINVAL;
+  if (dev_pool && (reinterpret_cast<uintptr_t>(dev_pool) & 255)) return CS_EINVAL;
+  cs_kv* kv = new (std::nothrow) cs_kv();
+  if (!kv) return CS_ENOMEM;
+  kv->model = m;
+  kv->num_pages = num_pages;
+  kv->page_size = page_size;
+  kv->max_seqs = max_seqs;
+  kv->max_pages_per_seq = max_pages_per_seq;
+  kv->plane_elems = static_cast<size_t>(num_pages) * m->d.n_kv_heads * page_size * m->d.head_dim;
+  kv->ctx_len.assign(max_seqs, -1);
+  kv->n_pages.assign(max_seqs, 0);
+  const uint64_t bytes = cs_kv_pool_bytes(m, num_pages, page_size);
+  int rc = CS_OK;
+  cudaError_t e;
+  if (dev_pool) {
+    kv->pool = static_cast<uint16_t*>(dev_pool);
+  } else {
+    void* p = nullptr;
+    e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc(kv pool)"); cs_kv_free(kv); return rc; }
+    kv->pool = static_cast<uint16_t*>(p);
+    kv->own_pool = true;
+    e = cudaMemset(p, 0, bytes);
+    if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMemset(kv pool)"); cs_kv_free(kv); return rc; }
+  }
+  const size_t tbytes = sizeof(int32_t) * static_cast<size_t>(max_seqs) * max_pages_per_seq;
+  e = cudaMallocHost(reinterpret_cast<void**>(&kv->table_host), tbytes);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&kv->table_dev), tbytes);
+  if (e == cudaSuccess) e = cudaMemset(kv->table_dev, 0, tbytes);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&kv->upload_ev, cudaEventDisableTiming);
+  if (e != cudaSuccess) { rc = cuda_fail(e, "kv page table"); cs_kv_free(kv); return rc; }
+  std::memset(kv->table_host, 0, tbytes);
+  if (!make_tensor_map_bf16(&kv->tm_pool, kv->pool, rows, m->d.head_dim, kPageSize, 64, true)) {
+    g_cuda_error = "cuTensorMapEncodeTiled failed for the kv pool";
+    cs_kv_free(kv);
+    return CS_ECUDA;
+  }
+  *out = kv;
+  return CS_OK;
+}
+
+int cs_kv_free(cs_kv* kv) {
+  if (!kv) return CS_OK;
+  cudaDeviceSynchronize();
+  if (kv->own_pool && kv->pool) cudaFree(kv->pool);
+  if (kv->table_host) cudaFreeHost(kv->table_host);
+  if (kv->table_dev) cudaFree(kv->table_dev);
+  if (kv->upload_ev) cudaEventDestroy(kv->upload_ev);
+  kv->fill_tmp.release();
+  delete kv;
+  return CS_OK;
+}
+
+int cs_kv_set_seq(cs_kv* kv, int seq, const int32_t* page_ids, int n_pages, int ctx_len) {
+  if (!kv || seq < 0 || seq >= kv->max_seqs || n_pages < 0 || n_pages > kv->max_pages_per_seq || ctx_len < 0 ||
+      ctx_len > n_pages * kv->page_size || (n_pages > 0 && !page_ids))
+    return CS_EINVAL;
+  for (int i = 0; i < n_pages; ++i)
+    if (page_ids[i] < 0 || page_ids[i] >= kv->num_pages) return CS_EINVAL;
+  if (kv->upload_pending) {
+    CS_CUDA(cudaEventSynchronize(kv->upload_ev));
+    kv->upload_pending = false;
+  }
+  int32_t* row = kv->table_host + static_cast<size_t>(seq) * kv->max_pages_per_seq;
+  for (int i = 0; i < n_pages; ++i) row[i] = page_ids[i];
+  kv->ctx_len[seq] = ctx_len;
+  kv->n_pages[seq] = n_pages;
+  kv->dirty = true;
+  return CS_OK;
+}
+
+int cs_kv_fill(cs_kv* kv, int seq, int layer, const uint16_t* host_k, const uint16_t* host_v, void* stream) {
+  if (!kv || seq < 0 || seq >= kv->max_seqs || layer < 0 || layer >= kv->model->d.n_layers) return CS_EINVAL;
+  if (kv->ctx_len[seq] < 0) return CS_ESTATE;
+  const int c = kv->ctx_len[seq];
+  if (c == 0) return CS_OK;
+  if (!host_k || !host_v) return CS_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const cs_model_desc& d = kv->model->d;
+  const size_t row = static_cast<size_t>(d.n_kv_heads) * d.head_dim;
+  const size_t elems = static_cast<size_t>(c) * row;
+  int rc;
+  if ((rc = kv->fill_tmp.ensure(2 * elems * 2))) return rc;
+  if ((rc = upload_table(kv, s))) return rc;
+  uint16_t* tk = static_cast<uint16_t*>(kv->fill_tmp.p);
+  uint16_t* tv = tk + elems;
+  CS_CUDA(cudaMemcpyAsync(tk, host_k, elems * 2, cudaMemcpyHostToDevice, s));
+  CS_CUDA(cudaMemcpyAsync(tv, host_v, elems * 2, cudaMemcpyHostToDevice, s));
+  CS_CUDA(launch_kv_scatter(tk, tv, static_cast<int>(row), nullptr, nullptr, seq, 0, kv->table_dev,
+                            kv->max_pages_per_seq, kv->pool + static_cast<size_t>(2 * layer) * kv->plane_elems,
+                            kv->pool + static_cast<size_t>(2 * layer + 1) * kv->plane_elems, d.n_kv_heads, d.head_dim,
+                            kPageSize, c, s));
+  CS_CUDA(cudaStreamSynchronize(s));
+  return CS_OK;
+}
+
+int cs_prefill(cs_model* m, cs_kv* kv, const int32_t* seq_ids, const int32_t* tokens, const int32_t* lens, int B,
+               void* stream) {
+  if (!m || !kv || kv->model != m || B < 0) return CS_EINVAL;
+  if (B == 0) return CS_OK;
+  if (!seq_ids || !tokens || !lens) return CS_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  for (int i = 0; i < B; ++i) {
+    if (seq_ids[i] < 0 || seq_ids[i] >= kv->max_seqs || lens[i] < 1) return CS_EINVAL;
+    if (kv->ctx_len[seq_ids[i]] < 0) return CS_ESTATE;
+    if (kv->ctx_len[seq_ids[i]] + lens[i] > kv->n_pages[seq_ids[i]] * kv->page_size) return CS_EINVAL;
+    for (int j = 0; j < i; ++j)
+      if (seq_ids[j] == seq_ids[i]) return CS_EINVAL;
+  }
+  int rc;
+  BatchLayout L;
+  const int32_t *dev_meta, *dev_tok;
+  if ((rc = stage_batch(m, kv, seq_ids, B, tokens, 0, lens, &L, &dev_meta, &dev_tok, s))) return rc;
+  if ((rc = upload_table(kv, s))) return rc;
+  if ((rc = run_layers(m, kv, kv, L, dev_meta, dev_tok, s))) return rc;
+  for (int i = 0; i < B; ++i) kv->ctx_len[seq_ids[i]] += lens[i];
+  return CS_OK;
+}
+
+int cs_verify_steps(cs_model* m, const cs_kv* ckv, const int32_t* seq_ids, int B, const int32_t* step_tokens,
+                    int tokens_on_device, const int32_t* step_lens, const int32_t* verdict_ids, int n_verdict,
+                    float tau, float* out_conf, uint8_t* out_accept, int32_t* out_verdict, void* stream) {
+  if (!m || !ckv || ckv->model != m || B < 0) return CS_EINVAL;
+  if (tau != tau) return CS_EINVAL;
+  if (n_verdict < 1 || n_verdict > 8 || !verdict_ids) return CS_EINVAL;
+  for (int j = 0; j < n_verdict; ++j)
+    if (verdict_ids[j] < 0 || verdict_ids[j] >= m->d.vocab) return CS_EINVAL;
+  if (B == 0) return CS_OK;
+  if (!seq_ids || !step_tokens || !step_lens || !out_conf || !out_accept) return CS_EINVAL;
+  cs_kv* kv = const_cast<cs_kv*>(ckv);  // only the upload bookkeeping of the page table changes
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc;
+  BatchLayout L;
+  const int32_t *dev_meta, *dev_tok;
+  if ((rc = stage_batch(m, kv, seq_ids, B, step_tokens, tokens_on_device, step_lens, &L, &dev_meta, &dev_tok, s)))
+    return rc;
+  if ((rc = upload_table(kv, s))) return rc;
+  if ((rc = run_layers(m, kv, nullptr, L, dev_meta, dev_tok, s))) return rc;
+
+  const cs_model_desc& d = m->d;
+  float* x = static_cast<float*>(m->x.p);
+  uint16_t* h_last = static_cast<uint16_t*>(m->h_last.p);
+  const int B_all = ((B + 63) / 64) * 64;
+  CS_CUDA(launch_last_rows_norm(x, dev_meta + L.off_cu, m->final_norm, h_last, B, B_all, d.d_model, d.rms_eps, s));
+  CUtensorMap tm_h;
+  int tiles_per_cta;
+  const int grid = lm_head_grid(d.vocab, &tiles_per_cta);
+  for (int b0 = 0; b0 < B; b0 += 64) {
+    const int bc = std::min(64, B - b0);
+    const int bp = lm_head_batch_pad(bc);
+    if (!make_tensor_map_bf16(&tm_h, h_last, B_all, d.d_model, bp, 64, true)) {
+      g_cuda_error = "cuTensorMapEncodeTiled failed for the last-position hidden states";
+      return CS_ECUDA;
+    }
+    float* part_max = static_cast<float*>(m->lm_part.p) + static_cast<size_t>(b0 / 64) * 2 * kNumSMs * 64;
+    float* part_sum = part_max + kNumSMs * 64;
+    float* vlog = static_cast<float*>(m->vlogits.p) + static_cast<size_t>(b0) * 8;
+    float* logits = m->keep_logits ? static_cast<float*>(m->logits.p) + static_cast<size_t>(b0) * d.vocab : nullptr;
+    CS_CUDA(launch_lm_head(m->tm_lm, tm_h, b0, bc, bp, d.d_model, d.vocab, verdict_ids, n_verdict, part_max, part_sum,
+                           vlog, logits, m->status, s));
+    CS_CUDA(launch_gate(part_max, part_sum, grid, bp, vlog, n_verdict, bc, tau, out_conf + b0, out_accept + b0,
+                        out_verdict ? out_verdict + b0 : nullptr, static_cast<float*>(m->lse.p) + b0, s));
+  }
+  m->last_B = B;
+  return CS_OK;
+}
+
+int cs_escalate_mask(const float* conf, int B, float tau, uint8_t* out_accept, int32_t* out_idx, int32_t* out_count,
+                     void* stream) {
+  if (B < 0 || B > 65536 || tau != tau || !out_count) return CS_EINVAL;
+  if (B > 0 && (!conf || !out_idx)) return CS_EINVAL;
+  CS_CUDA(launch_escalate(conf, B, tau, out_accept, out_idx, out_count, static_cast<cudaStream_t>(stream)));
+  return CS_OK;
+}
+
+int cs_set_keep_logits(cs_model* m, int keep) {
+  if (!m) return CS_EINVAL;
+  m->keep_logits = keep != 0;
+  return CS_OK;
+}
+
+int cs_get_last_logits(cs_model* m, float* dev_out, int B, void* stream) {
+  if (!m || !dev_out || B < 1) return CS_EINVAL;
+  if (!m->keep_logits || B > m->last_B || !m->logits.p) return CS_ESTATE;
+  CS_CUDA(cudaMemcpyAsync(dev_out, m->logits.p, static_cast<size_t>(B) * m->d.vocab * 4, cudaMemcpyDeviceToDevice,
+                          static_cast<cudaStream_t>(stream)));
+  return CS_OK;
+}
+
+int cs_get_last_lse(cs_model* m, float* dev_out, int B, void* stream) {
+  if (!m || !dev_out || B < 1) return CS_EINVAL;
+  if (B > m->last_B || !m->lse.p) return CS_ESTATE;
+  CS_CUDA(cudaMemcpyAsync(dev_out, m->lse.p, static_cast<size_t>(B) * 4, cudaMemcpyDeviceToDevice,
+                          static_cast<cudaStream_t>(stream)));
+  return CS_OK;
+}
+
+int cs_last_status(cs_model* m, void* stream) {
+  if (!m) return CS_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint32_t v = 0;
+  CS_CUDA(cudaMemcpyAsync(&v, m->status, 4, cudaMemcpyDeviceToHost, s));
+  CS_CUDA(cudaStreamSynchronize(s));
+  if (v) CS_CUDA(cudaMemsetAsync(m->status, 0, 4, s));
+  return (v & 1u) ? CS_ETIMEOUT : CS_OK;
+}
+
+int cs_gemm_bf16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* out, int M, int N, int K,
+                 int epilogue, void* stream) {
+  if (!a || !w || !out || M < 0 || N < 8 || K < 8 || (N % 8) || (K % 8) || epilogue < 0 || epilogue > 2)
+    return CS_EINVAL;
+  if (epilogue == kEpiSwiGLU && !w2) return CS_EINVAL;
+  if (M == 0) return CS_OK;
+  if (!g_test_status) {
+    CS_CUDA(cudaMalloc(reinterpret_cast<void**>(&g_test_status), 256));
+    CS_CUDA(cudaMemset(g_test_status, 0, 256));
+  }
+  CUtensorMap ta, tb, tb2;
+  if (!make_gemm_operand_map(&ta, a, M, K) || !make_gemm_operand_map(&tb, w, N, K) ||
+      (w2 && !make_gemm_operand_map(&tb2, w2, N, K))) {
+    g_cuda_error = "cuTensorMapEncodeTiled failed";
+    return CS_ECUDA;
+  }
+  CS_CUDA(gemm_bf16(ta, tb, w2 ? &tb2 : nullptr, out, M, N, K, epilogue, g_test_status,
+                    static_cast<cudaStream_t>(stream)));
+  return CS_OK;
+}
+
+int cs_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps, void* stream) {
+  if (!x || !gain || !out || rows < 0 || d < 4 || (d % 4)) return CS_EINVAL;
+  CS_CUDA(launch_rmsnorm(x, gain, out, rows, d, eps, static_cast<cudaStream_t>(stream)));
+  return CS_OK;
+}
+
+}  // extern "C"

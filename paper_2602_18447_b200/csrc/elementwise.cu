@@ -1,0 +1,162 @@
+// Memory-bound pieces of the decoder layers: embedding gather, RMSNorm, rotary tables and rotation,
+// and the scatter of K/V rows into cache pages.
+#include "kernels.h"
+
+#include "common.cuh"
+
+namespace cs {
+
+namespace {
+
+thread_local int64_t g_launches = 0;
+
+__global__ void embed_kernel(const int32_t* __restrict__ tokens, const uint16_t* __restrict__ embed,
+                             float* __restrict__ x, int T, int d, int vocab) {
+  const int t = blockIdx.x;
+  int tok = tokens[t];
+  tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);
+  const uint4* src = reinterpret_cast<const uint4*>(embed + static_cast<size_t>(tok) * d);
+  float4* dst = reinterpret_cast<float4*>(x + static_cast<size_t>(t) * d);
+  for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
+    const uint4 v = src[i];
+    dst[2 * i] = make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
+    dst[2 * i + 1] = make_float4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w));
+  }
+}
+
+// One warp per row: sum of squares, then scale and round to bf16. The second pass re-reads the row from L2.
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
+                               uint16_t* __restrict__ out, int rows, int d, float eps) {
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(row) * d);
+  float ss = 0.f;
+  for (int i = lane; i < d / 4; i += 32) {
+    const float4 v = xr[i];
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = warp_sum(ss);
+  const float r = rsqrtf(ss / static_cast<float>(d) + eps);
+  const float4* g4 = reinterpret_cast<const float4*>(gain);
+  uint2* o = reinterpret_cast<uint2*>(out + static_cast<size_t>(row) * d);
+  for (int i = lane; i < d / 4; i += 32) {
+    const float4 v = xr[i];
+    const float4 g = g4[i];
+    o[i] = make_uint2(pack_bf16x2(v.x * r * g.x, v.y * r * g.y), pack_bf16x2(v.z * r * g.z, v.w * r * g.w));
+  }
+}
+
+__global__ void rope_table_kernel(const int32_t* __restrict__ pos, const double* __restrict__ inv_freq,
+                                  float2* __restrict__ table, int T, int half) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= T * half) return;
+  const int t = i / half, j = i - t * half;
+  double s, c;
+  sincos(static_cast<double>(pos[t]) * inv_freq[j], &s, &c);
+  table[i] = make_float2(static_cast<float>(c), static_cast<float>(s));
+}
+
+// Thread per (row, head, pair of adjacent rotation pairs): elements j, j+1 and j+half, j+half+1.
+__global__ void rope_apply_kernel(uint16_t* __restrict__ qkv, const float2* __restrict__ table, int T, int n_qkv,
+                                  int n_rot_heads, int hd) {
+  const int half = hd >> 1;
+  const int per_row = n_rot_heads * (half >> 1);
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= T * per_row) return;
+  const int t = i / per_row;
+  const int r = i - t * per_row;
+  const int head = r / (half >> 1);
+  const int j = (r - head * (half >> 1)) * 2;
+  uint32_t* lo = reinterpret_cast<uint32_t*>(qkv + static_cast<size_t>(t) * n_qkv + head * hd + j);
+  uint32_t* hi = reinterpret_cast<uint32_t*>(qkv + static_cast<size_t>(t) * n_qkv + head * hd + half + j);
+  const uint32_t a = *lo, b = *hi;
+  const float2 cs0 = table[t * half + j], cs1 = table[t * half + j + 1];
+  const float a0 = bf16_lo(a), a1 = bf16_hi(a), b0 = bf16_lo(b), b1 = bf16_hi(b);
+  *lo = pack_bf16x2(a0 * cs0.x - b0 * cs0.y, a1 * cs1.x - b1 * cs1.y);
+  *hi = pack_bf16x2(b0 * cs0.x + a0 * cs0.y, b1 * cs1.x + a1 * cs1.y);
+}
+
+// Thread per 16 bytes of a K row and of a V row.
+__global__ void kv_scatter_kernel(const uint16_t* __restrict__ src_k, const uint16_t* __restrict__ src_v,
+                                  int row_stride, const int32_t* __restrict__ tok_seq,
+                                  const int32_t* __restrict__ tok_pos, int const_seq, int pos0,
+                                  const int32_t* __restrict__ page_table,
+                                  int max_pages_per_seq, uint16_t* __restrict__ pool_k, uint16_t* __restrict__ pool_v,
+                                  int n_kv_heads, int hd, int page_size, int T) {
+  const int chunks = n_kv_heads * hd / 8;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= T * chunks) return;
+  const int t = i / chunks;
+  const int c = i - t * chunks;
+  const int head = (c * 8) / hd;
+  const int e = c * 8 - head * hd;
+  const int pos = tok_seq ? tok_pos[t] : pos0 + t;
+  const int seq = tok_seq ? tok_seq[t] : const_seq;
+  const int page = page_table[static_cast<size_t>(seq) * max_pages_per_seq + pos / page_size];
+  const int slot = pos % page_size;
+  const size_t dst = ((static_cast<size_t>(page) * n_kv_heads + head) * page_size + slot) * hd + e;
+  const size_t src = static_cast<size_t>(t) * row_stride + c * 8;
+  *reinterpret_cast<uint4*>(pool_k + dst) = *reinterpret_cast<const uint4*>(src_k + src);
+  *reinterpret_cast<uint4*>(pool_v + dst) = *reinterpret_cast<const uint4*>(src_v + src);
+}
+
+}  // namespace
+
+void count_launch(int n) { g_launches += n; }
+int64_t take_launch_count() {
+  const int64_t v = g_launches;
+  g_launches = 0;
+  return v;
+}
+
+cudaError_t launch_embed(const int32_t* tokens, const uint16_t* embed, float* x, int T, int d, int vocab,
+                         cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  embed_kernel<<<T, 128, 0, s>>>(tokens, embed, x, T, d, vocab);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps,
+                           cudaStream_t s) {
+  if (rows <= 0) return cudaSuccess;
+  const int warps = 8;
+  rmsnorm_kernel<<<(rows + warps - 1) / warps, warps * 32, 0, s>>>(x, gain, out, rows, d, eps);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rope_table(const int32_t* pos, const double* inv_freq, float2* table, int T, int half,
+                              cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  const int n = T * half;
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(pos, inv_freq, table, T, half);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rope_apply(uint16_t* qkv, const float2* table, int T, int n_qkv, int n_rot_heads, int hd,
+                              cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  const int n = T * n_rot_heads * (hd / 4);
+  rope_apply_kernel<<<(n + 255) / 256, 256, 0, s>>>(qkv, table, T, n_qkv, n_rot_heads, hd);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int row_stride, const int32_t* tok_seq,
+                              const int32_t* tok_pos, int const_seq, int pos0, const int32_t* page_table,
+                              int max_pages_per_seq,
+                              uint16_t* pool_k_plane, uint16_t* pool_v_plane, int n_kv_heads, int hd, int page_size,
+                              int T, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  const int n = T * n_kv_heads * hd / 8;
+  kv_scatter_kernel<<<(n + 255) / 256, 256, 0, s>>>(src_k, src_v, row_stride, tok_seq, tok_pos, const_seq, pos0, page_table,
+                                                    max_pages_per_seq, pool_k_plane, pool_v_plane, n_kv_heads, hd,
+                                                    page_size, T);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace cs

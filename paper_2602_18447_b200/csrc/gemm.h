@@ -1,0 +1,25 @@
+// Host interface of the tcgen05 projection GEMM.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cs {
+
+enum GemmEpilogue {
+  kEpiStoreBf16 = 0,  // out bf16 [M,N] = a * w^T
+  kEpiResidAdd = 1,   // out fp32 [M,N] += a * w^T   (atomic adds, k-range split over the SMs)
+  kEpiSwiGLU = 2      // out bf16 [M,N] = silu(a * w^T) * (a * w2^T)
+};
+
+// 2D bf16 tensor map over a row-major [rows, cols] matrix; box = [box_rows, box_cols].
+bool make_tensor_map_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                          uint32_t box_cols, bool swizzle128);
+// Tensor map of a GEMM operand ([rows, k] bf16, K-major): 128-row x 64-column boxes, 128-byte swizzle.
+bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k);
+
+cudaError_t gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,
+                      int K, int epilogue, uint32_t* status, cudaStream_t stream);
+
+}  // namespace cs

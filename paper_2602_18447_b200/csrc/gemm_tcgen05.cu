@@ -1,0 +1,345 @@
+// Projection GEMMs of the decoder layers: out = a[M,K] * w[N,K]^T, bf16 in, fp32 accumulate in TMEM.
+//
+// One persistent CTA per SM. Warp 0 feeds a ring of shared-memory stages with TMA (128-byte swizzle), warp 1
+// issues tcgen05.mma into one of two TMEM accumulators, warps 2-5 drain the other accumulator (tcgen05.ld)
+// and apply the epilogue, so the epilogue of one tile overlaps the main loop of the next.
+//
+// Work is measured in k-blocks (128 x BN x 64 products). Each CTA owns a contiguous range of k-blocks in the
+// order (n tile, m tile, k); a range may start or end inside a tile. For the two epilogues that need the whole
+// sum (bf16 store, SwiGLU) the ranges are whole tiles. For the residual epilogue (x += a * w^T, fp32) the
+// range is cut evenly over the SMs whatever the tile boundaries are, and every piece is added into x with
+// vector atomics, which is what lets the narrow O and down projections fill all SMs.
+#include "gemm.h"
+
+#include "kernels.h"
+
+#include "common.cuh"
+
+namespace cs {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int kGemmThreads = 192;
+constexpr int kABytes = BM * BK * 2;
+
+template <int BN>
+struct GemmSmem {
+  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kBarBytes = 256;
+  static constexpr int kTotal = kStages * kStageBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
+};
+
+struct Segment {
+  int tile, kb0, len;
+};
+
+__device__ __forceinline__ Segment next_segment(int u, int end, int kblocks) {
+  Segment s;
+  s.tile = u / kblocks;
+  s.kb0 = u - s.tile * kblocks;
+  s.len = min(kblocks - s.kb0, end - u);
+  return s;
+}
+
+__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void st_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                 const __grid_constant__ CUtensorMap tm_b2, void* __restrict__ out, int M, int N, int m_tiles,
+                 int kblocks, int total_units, int units_per_cta, uint32_t* status) {
+  using L = GemmSmem<BN>;
+  constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
+  constexpr uint32_t kTmemCols = 2 * BN;
+  constexpr uint32_t kIdesc = umma_idesc_bf16(BM, BN);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kStages * L::kStageBytes);
+  uint64_t* full_bar = bars;                       // [kStages] TMA -> MMA
+  uint64_t* empty_bar = bars + L::kStages;         // [kStages] MMA -> TMA
+  uint64_t* acc_full = bars + 2 * L::kStages;      // [2] MMA -> epilogue
+  uint64_t* acc_empty = bars + 2 * L::kStages + 2; // [2] epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * L::kStages + 4);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  const int start = blockIdx.x * units_per_cta;
+  const int end = min(total_units, start + units_per_cta);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < L::kStages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&acc_full[a], 1);
+      mbar_init(&acc_empty[a], 4);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&tm_a);
+    tma_prefetch_desc(&tm_b);
+    if (EPI == kEpiSwiGLU) tma_prefetch_desc(&tm_b2);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int u = start; u < end && ok;) {
+        const Segment sg = next_segment(u, end, kblocks);
+        const int m0 = (sg.tile % m_tiles) * BM;
+        const int n0 = (sg.tile / m_tiles) * OUT_BN;
+        for (int kb = sg.kb0; kb < sg.kb0 + sg.len; ++kb) {
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
+          uint8_t* sa = smem + stage * L::kStageBytes;
+          uint8_t* sb = sa + kABytes;
+          mbar_arrive_expect_tx(&full_bar[stage], L::kStageBytes);
+          tma_load_2d(sa, &tm_a, &full_bar[stage], kb * BK, m0);
+          if (EPI == kEpiSwiGLU) {
+            tma_load_2d(sb, &tm_b, &full_bar[stage], kb * BK, n0);
+            tma_load_2d(sb + 128 * BK * 2, &tm_b2, &full_bar[stage], kb * BK, n0);
+          } else {
+#pragma unroll
+            for (int h = 0; h < BN / 128; ++h)
+              tma_load_2d(sb + h * 128 * BK * 2, &tm_b, &full_bar[stage], kb * BK, n0 + h * 128);
+          }
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+        u += sg.len;
+      }
+      // In a healthy run the MMA warp has waited for every copy before the CTA exits. After an abort, give
+      // the copies still in flight time to land in shared memory before the CTA may go away.
+      if (!ok)
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int u = start; u < end && ok;) {
+        const Segment sg = next_segment(u, end, kblocks);
+        if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int i = 0; i < sg.len; ++i) {
+          if (!mbar_wait(&full_bar[stage], phase, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint64_t adesc = umma_desc_k128(sa);
+          const uint64_t bdesc = umma_desc_k128(sa + kABytes);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)
+            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (i | k) != 0);
+          umma_commit(&empty_bar[stage]);
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(&acc_full[acc]);
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+        u += sg.len;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quad = warp & 3;  // the TMEM lane quadrant this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int u = start; u < end && ok;) {
+      const Segment sg = next_segment(u, end, kblocks);
+      const int m0 = (sg.tile % m_tiles) * BM;
+      const int n0 = (sg.tile / m_tiles) * OUT_BN;
+      if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, status)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
+      const int row = m0 + quad * 32 + lane;
+      const bool row_ok = row < M;
+      uint32_t r[32];
+      if (EPI == kEpiSwiGLU) {
+        uint32_t r2[32];
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + static_cast<size_t>(row) * N;
+#pragma unroll 1
+        for (int c = 0; c < OUT_BN / 32; ++c) {
+          tmem_ld_32x32(t_row + c * 32, r);
+          tmem_ld_32x32(t_row + OUT_BN + c * 32, r2);
+          tmem_ld_wait();
+          uint32_t p[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float g0 = __uint_as_float(r[2 * j]), g1 = __uint_as_float(r[2 * j + 1]);
+            const float u0 = __uint_as_float(r2[2 * j]), u1 = __uint_as_float(r2[2 * j + 1]);
+            p[j] = pack_bf16x2(silu_f(g0) * u0, silu_f(g1) * u1);
+          }
+          const int col = n0 + c * 32;
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (col + j * 8 < N) st_v4(o + col + j * 8, p[4 * j], p[4 * j + 1], p[4 * j + 2], p[4 * j + 3]);
+          }
+        }
+      } else if (EPI == kEpiStoreBf16) {
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + static_cast<size_t>(row) * N;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          tmem_ld_32x32(t_row + c * 32, r);
+          tmem_ld_wait();
+          const int col = n0 + c * 32;
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (col + j * 8 < N)
+                st_v4(o + col + j * 8, pack_bf16x2(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1])),
+                      pack_bf16x2(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3])),
+                      pack_bf16x2(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5])),
+                      pack_bf16x2(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7])));
+          }
+        }
+      } else {
+        float* o = reinterpret_cast<float*>(out) + static_cast<size_t>(row) * N;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          tmem_ld_32x32(t_row + c * 32, r);
+          tmem_ld_wait();
+          const int col = n0 + c * 32;
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (col + j * 4 < N)
+                red_add_v4(o + col + j * 4, __uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                           __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+      u += sg.len;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+template <int BN, int EPI>
+cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, void* out, int M, int N,
+                   int K, uint32_t* status, cudaStream_t stream) {
+  using L = GemmSmem<BN>;
+  constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int m_tiles = (M + BM - 1) / BM;
+  const int n_tiles = (N + OUT_BN - 1) / OUT_BN;
+  const int kblocks = (K + BK - 1) / BK;
+  const int tiles = m_tiles * n_tiles;
+  const int total = tiles * kblocks;
+  int grid, upc;
+  if (EPI == kEpiResidAdd) {
+    grid = total < kNumSMs ? total : kNumSMs;
+    upc = (total + grid - 1) / grid;
+    grid = (total + upc - 1) / upc;
+  } else {
+    const int tpc = (tiles + kNumSMs - 1) / kNumSMs;
+    grid = (tiles + tpc - 1) / tpc;
+    upc = tpc * kblocks;
+  }
+  gemm_bf16_kernel<BN, EPI><<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tb, tb2, out, M, N, m_tiles, kblocks, total,
+                                                                      upc, status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool make_tensor_map_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                          uint32_t box_cols, bool swizzle128) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k) {
+  return make_tensor_map_bf16(tm, base, static_cast<uint64_t>(rows), static_cast<uint64_t>(k), 128, 64, true);
+}
+
+cudaError_t gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,
+                      int K, int epilogue, uint32_t* status, cudaStream_t stream) {
+  if (M <= 0) return cudaSuccess;
+  switch (epilogue) {
+    case kEpiStoreBf16:
+      // Narrow outputs get 128-wide tiles so that the tile count comes closer to the SM count.
+      if (((M + 127) / 128) * ((N + 255) / 256) < kNumSMs / 2 + 20)
+        return launch<128, kEpiStoreBf16>(ta, tb, tb, out, M, N, K, status, stream);
+      return launch<256, kEpiStoreBf16>(ta, tb, tb, out, M, N, K, status, stream);
+    case kEpiResidAdd:
+      return launch<256, kEpiResidAdd>(ta, tb, tb, out, M, N, K, status, stream);
+    case kEpiSwiGLU:
+      return launch<256, kEpiSwiGLU>(ta, tb, *tb2, out, M, N, K, status, stream);
+    default:
+      return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace cs

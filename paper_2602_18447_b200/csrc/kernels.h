@@ -1,0 +1,92 @@
+// Launchers of the non-GEMM kernels of the verification pass. All are asynchronous on `stream`.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cs {
+
+constexpr int kNumSMs = 148;
+
+// One unit of attention work: a tile of 64 query rows of one (step, kv head) over a range of 64-key tiles.
+// Query rows of a (step, kv head) are the pairs (new position p, head-in-group g) flattened as p * G + g.
+// Key tiles 0 .. ctx_tiles-1 cover the cached context (4 pages each), the following ones the step's own
+// new keys.
+struct AttnItem {
+  int32_t step;       // index into the batch
+  int32_t kv_head;
+  int32_t q_row0;     // first flattened query row of the tile (multiple of 64)
+  int32_t tile_begin; // key tile range [tile_begin, tile_end)
+  int32_t tile_end;
+  int32_t slot;       // partial-result slot, or -1 when the range is the whole key sequence
+  int32_t pad0, pad1;
+};
+
+// A group of partial results to merge: slots [slot0, slot0 + n_splits) belong to one query tile.
+struct AttnMerge {
+  int32_t step, kv_head, q_row0, slot0, n_splits, pad0, pad1, pad2;
+};
+
+struct AttnParams {
+  const uint16_t* qkv;      // [T, n_qkv] bf16: q heads, k heads, v heads (q, k already rotated)
+  uint16_t* out;            // [T, Hq*hd] bf16
+  const int32_t* cu_new;    // [B+1]
+  const int32_t* ctx_len;   // [B]
+  const int32_t* seq_id;    // [B]
+  const int32_t* page_table;// [max_seqs, max_pages_per_seq]
+  int32_t max_pages_per_seq;
+  int32_t n_q_heads, n_kv_heads, head_dim, n_qkv;
+  int32_t k_row_base, v_row_base;  // first pool row of this layer's K and V planes
+  float scale_log2e;        // log2(e) / sqrt(head_dim)
+  float* part_o;            // [slots, 64, hd] unnormalised partial outputs
+  float* part_ml;           // [slots, 64, 2]  running max (raw score units) and sum
+  uint32_t* status;
+};
+
+cudaError_t launch_embed(const int32_t* tokens, const uint16_t* embed, float* x, int T, int d, int vocab,
+                         cudaStream_t s);
+cudaError_t launch_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps,
+                           cudaStream_t s);
+// cos/sin of pos[t] * inv_freq[j] in double, stored as float2 [T, half].
+cudaError_t launch_rope_table(const int32_t* pos, const double* inv_freq, float2* table, int T, int half,
+                              cudaStream_t s);
+// Rotate the first n_rot_heads heads (q heads then k heads) of every row of qkv in place.
+cudaError_t launch_rope_apply(uint16_t* qkv, const float2* table, int T, int n_qkv, int n_rot_heads, int hd,
+                              cudaStream_t s);
+// Copy K and V rows into cache pages. src rows are [n_kv_heads*hd] wide at src_k/src_v + t*row_stride.
+// Row t goes to sequence tok_seq[t], position tok_pos[t]; when tok_seq is NULL, to sequence const_seq,
+// position pos0 + t.
+cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int row_stride, const int32_t* tok_seq,
+                              const int32_t* tok_pos, int const_seq, int pos0, const int32_t* page_table,
+                              int max_pages_per_seq,
+                              uint16_t* pool_k_plane, uint16_t* pool_v_plane, int n_kv_heads, int hd, int page_size,
+                              int T, cudaStream_t s);
+
+cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_pool, const CUtensorMap& tm_qkv,
+                             const AttnItem* items, int n_items, const AttnMerge* merges, int n_merges,
+                             cudaStream_t s);
+
+// h[b] = RMSNorm(x[last_row[b]]) as bf16 [B_pad, d]; rows B..B_pad-1 are zeroed.
+cudaError_t launch_last_rows_norm(const float* x, const int32_t* cu_new, const float* gain, uint16_t* h, int B,
+                                  int B_pad, int d, float eps, cudaStream_t s);
+// LM head over 128-row vocabulary tiles (tcgen05): per CTA and step the maximum and the sum of exp(z - max)
+// of the CTA's rows, the logits of the verdict ids, and optionally all logits. h rows [h_row0, h_row0 + B_pad)
+// of the tensor map tm_h are the batch; B_pad is 16, 32 or 64. part_max / part_sum are [grid, B_pad].
+cudaError_t launch_lm_head(const CUtensorMap& tm_w, const CUtensorMap& tm_h, int h_row0, int B, int B_pad, int d,
+                           int vocab, const int32_t* verdict_ids_host, int n_verdict, float* part_max,
+                           float* part_sum, float* verdict_logits, float* logits_or_null, uint32_t* status,
+                           cudaStream_t s);
+int lm_head_grid(int vocab, int* tiles_per_cta);
+int lm_head_batch_pad(int B);
+// Merge the CTAs' pairs, form the confidence and apply the threshold.
+cudaError_t launch_gate(const float* part_max, const float* part_sum, int n_slices, int nb_stride,
+                        const float* verdict_logits, int n_verdict, int B, float tau, float* out_conf,
+                        uint8_t* out_accept, int32_t* out_verdict, float* out_lse, cudaStream_t s);
+cudaError_t launch_escalate(const float* conf, int B, float tau, uint8_t* out_accept, int32_t* out_idx,
+                            int32_t* out_count, cudaStream_t s);
+
+void count_launch(int n = 1);
+int64_t take_launch_count();
+
+}  // namespace cs

@@ -1,0 +1,396 @@
+// Last-position LM head with the logsumexp over the vocabulary fused in, and the confidence gate.
+//
+// logits^T[V, B] = W_lm[V, d] * h[B, d]^T is a weight-streaming product (B is 8..64): each CTA walks over
+// 128-row tiles of W_lm, brought in by TMA, multiplies them on the tensor cores (tcgen05, M = 128 vocabulary
+// rows, N = padded batch) and never writes the logits: every epilogue thread owns one TMEM lane (one
+// vocabulary row of each tile) and keeps, per step, a running maximum and a running sum of exp(z - max) over
+// the rows it has seen. At the end the 128 threads merge their pairs and the CTA emits one (max, sum) pair per
+// step; the gate kernel merges the CTAs' pairs, forms p = exp(z_verdict - lse) and applies the threshold.
+#include "kernels.h"
+
+#include "common.cuh"
+
+namespace cs {
+
+namespace {
+
+constexpr int kLmBM = 128;
+constexpr int kLmBK = 64;
+constexpr int kLmThreads = 192;
+constexpr int kLmWBytes = kLmBM * kLmBK * 2;
+constexpr int kLmMaxVerdict = 8;
+
+template <int NB>
+struct LmSmem {
+  static constexpr int kHBytes = NB * kLmBK * 2;
+  static constexpr int kStageBytes = kLmWBytes + ((kHBytes + 1023) / 1024) * 1024;
+  static constexpr int kStages = 8;
+  static constexpr int kBarOff = kStages * kStageBytes;
+  static constexpr int kRedOff = kBarOff + 256;                 // [4 warps][NB][2] floats
+  static constexpr int kTotal = kRedOff + 4 * NB * 2 * 4 + 1024;
+};
+
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+struct LmArgs {
+  int B, vocab, kblocks, n_tiles, tiles_per_cta, n_verdict, h_row0;
+  int verdict[kLmMaxVerdict];
+  float* part_max;        // [grid, NB]
+  float* part_sum;        // [grid, NB]
+  float* verdict_logits;  // [B, n_verdict]
+  float* logits;          // [B, vocab] or nullptr
+  uint32_t* status;
+};
+
+template <int NB>
+__global__ void __launch_bounds__(kLmThreads, 1)
+lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const LmArgs a) {
+  using L = LmSmem<NB>;
+  constexpr uint32_t kTmemCols = (2 * NB < 32) ? 32 : 2 * NB;
+  constexpr uint32_t kIdesc = umma_idesc_bf16(kLmBM, NB);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = bars + L::kStages;
+  uint64_t* acc_full = bars + 2 * L::kStages;
+  uint64_t* acc_empty = bars + 2 * L::kStages + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * L::kStages + 4);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* red = reinterpret_cast<float*>(smem + L::kRedOff);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile_begin = blockIdx.x * a.tiles_per_cta;
+  const int tile_end = min(a.n_tiles, tile_begin + a.tiles_per_cta);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < L::kStages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&acc_full[i], 1);
+      mbar_init(&acc_empty[i], 4);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&tm_w);
+    tma_prefetch_desc(&tm_h);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = tile_begin; t < tile_end && ok; ++t) {
+        for (int kb = 0; kb < a.kblocks; ++kb) {
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, a.status)) { ok = false; break; }
+          uint8_t* sw = smem + stage * L::kStageBytes;
+          mbar_arrive_expect_tx(&full_bar[stage], kLmWBytes + L::kHBytes);
+          tma_load_2d(sw, &tm_w, &full_bar[stage], kb * kLmBK, t * kLmBM);
+          tma_load_2d(sw + kLmWBytes, &tm_h, &full_bar[stage], kb * kLmBK, a.h_row0);
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok)
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int t = tile_begin; t < tile_end && ok; ++t) {
+        if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * NB;
+        for (int kb = 0; kb < a.kblocks; ++kb) {
+          if (!mbar_wait(&full_bar[stage], phase, abort_flag, a.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sw = smem_u32(smem + stage * L::kStageBytes);
+          const uint64_t adesc = umma_desc_k128(sw);
+          const uint64_t bdesc = umma_desc_k128(sw + kLmWBytes);
+#pragma unroll
+          for (int k = 0; k < kLmBK / 16; ++k)
+            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0);
+          umma_commit(&empty_bar[stage]);
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(&acc_full[acc]);
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    const int quad = warp & 3;
+    float run_m[NB], run_l[NB];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) { run_m[b] = -INFINITY; run_l[b] = 0.f; }
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int t = tile_begin; t < tile_end; ++t) {
+      if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, a.status)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + acc * NB + (static_cast<uint32_t>(quad * 32) << 16);
+      const int row = t * kLmBM + quad * 32 + lane;   // vocabulary id of this thread's lane
+      const bool row_ok = row < a.vocab;
+      uint32_t vmask = 0;   // which entries of verdict_ids name this row (an id may be listed twice)
+      for (int j = 0; j < a.n_verdict; ++j)
+        if (a.verdict[j] == row) vmask |= 1u << j;
+#pragma unroll
+      for (int c = 0; c < NB / 16; ++c) {
+        uint32_t r[16];
+        tmem_ld_32x16(t_row + c * 16, r);
+        tmem_ld_wait();
+        if (row_ok) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int b = c * 16 + j;
+            const float z = __uint_as_float(r[j]);
+            const float mn = fmaxf(run_m[b], z);
+            run_l[b] = run_l[b] * __expf(run_m[b] - mn) + __expf(z - mn);
+            run_m[b] = mn;
+            if (b < a.B) {
+              for (uint32_t vm = vmask; vm; vm &= vm - 1) a.verdict_logits[b * a.n_verdict + (__ffs(vm) - 1)] = z;
+              if (a.logits) a.logits[static_cast<size_t>(b) * a.vocab + row] = z;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    // Merge the per-thread pairs: across the warp by shuffles, across the four warps through shared memory.
+    if (ok) {
+#pragma unroll
+      for (int b = 0; b < NB; ++b) {
+        const float m = warp_max(run_m[b]);
+        const float l = warp_sum(run_m[b] == -INFINITY ? 0.f : run_l[b] * __expf(run_m[b] - m));
+        if (lane == 0) {
+          red[(quad * NB + b) * 2] = m;
+          red[(quad * NB + b) * 2 + 1] = l;
+        }
+      }
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (ok && quad == 0) {
+      for (int b = lane; b < NB; b += 32) {
+        float m = -INFINITY;
+        for (int q = 0; q < 4; ++q) m = fmaxf(m, red[(q * NB + b) * 2]);
+        float l = 0.f;
+        for (int q = 0; q < 4; ++q) {
+          const float mq = red[(q * NB + b) * 2];
+          l += (mq == -INFINITY) ? 0.f : red[(q * NB + b) * 2 + 1] * __expf(mq - m);
+        }
+        a.part_max[blockIdx.x * NB + b] = m;
+        a.part_sum[blockIdx.x * NB + b] = l;
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// One warp per step.
+__global__ void last_rows_norm_kernel(const float* __restrict__ x, const int32_t* __restrict__ cu_new,
+                                      const float* __restrict__ gain, uint16_t* __restrict__ h, int B, int B_pad,
+                                      int d, float eps) {
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B_pad) return;
+  uint2* o = reinterpret_cast<uint2*>(h + static_cast<size_t>(b) * d);
+  if (b >= B) {
+    for (int i = lane; i < d / 4; i += 32) o[i] = make_uint2(0u, 0u);
+    return;
+  }
+  const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(cu_new[b + 1] - 1) * d);
+  float ss = 0.f;
+  for (int i = lane; i < d / 4; i += 32) {
+    const float4 v = xr[i];
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = warp_sum(ss);
+  const float r = rsqrtf(ss / static_cast<float>(d) + eps);
+  const float4* g4 = reinterpret_cast<const float4*>(gain);
+  for (int i = lane; i < d / 4; i += 32) {
+    const float4 v = xr[i];
+    const float4 g = g4[i];
+    o[i] = make_uint2(pack_bf16x2(v.x * r * g.x, v.y * r * g.y), pack_bf16x2(v.z * r * g.z, v.w * r * g.w));
+  }
+}
+
+// One warp per step: merge the vocabulary slices, then confidence, decision and threshold (Eq. 4).
+__global__ void gate_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum, int n_slices,
+                            int nb_stride, const float* __restrict__ verdict_logits, int n_verdict, int B, float tau,
+                            float* __restrict__ out_conf, uint8_t* __restrict__ out_accept,
+                            int32_t* __restrict__ out_verdict, float* __restrict__ out_lse) {
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B) return;
+  float m = -INFINITY;
+  for (int s = lane; s < n_slices; s += 32) m = fmaxf(m, part_max[s * nb_stride + b]);
+  m = warp_max(m);
+  float l = 0.f;
+  for (int s = lane; s < n_slices; s += 32) {
+    const float ms = part_max[s * nb_stride + b];
+    if (ms != -INFINITY) l += part_sum[s * nb_stride + b] * expf(ms - m);
+  }
+  l = warp_sum(l);
+  if (lane == 0) {
+    const float lse = m + logf(l);
+    float best = -1.f;
+    int arg = 0;
+    bool nan = false;
+    for (int j = 0; j < n_verdict; ++j) {
+      const float pj = expf(verdict_logits[b * n_verdict + j] - lse);
+      if (pj != pj) nan = true;
+      if (pj > best) { best = pj; arg = j; }
+    }
+    const float conf = nan ? __int_as_float(0x7fc00000) : best;
+    out_conf[b] = conf;
+    out_accept[b] = (conf >= tau) ? 1 : 0;   // false for NaN: such a step is escalated
+    if (out_verdict) out_verdict[b] = arg;
+    if (out_lse) out_lse[b] = lse;
+  }
+}
+
+// Single CTA: flags, then an ordered compaction of the escalated indices by a block-wide scan.
+__global__ void escalate_kernel(const float* __restrict__ conf, int B, float tau, uint8_t* __restrict__ out_accept,
+                                int32_t* __restrict__ out_idx, int32_t* __restrict__ out_count) {
+  __shared__ int warp_tot[32];
+  __shared__ int base;
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  for (int i0 = 0; i0 < B; i0 += blockDim.x) {
+    const int i = i0 + threadIdx.x;
+    int esc = 0;
+    if (i < B) {
+      const int acc = (conf[i] >= tau) ? 1 : 0;
+      if (out_accept) out_accept[i] = static_cast<uint8_t>(acc);
+      esc = 1 - acc;
+    }
+    const unsigned ball = __ballot_sync(0xffffffffu, esc);
+    const int before = __popc(ball & ((1u << lane) - 1u));
+    if (lane == 0) warp_tot[warp] = __popc(ball);
+    __syncthreads();
+    int off = base;
+    for (int w = 0; w < warp; ++w) off += warp_tot[w];
+    if (esc) out_idx[off + before] = i;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int tot = 0;
+      for (int w = 0; w < nw; ++w) tot += warp_tot[w];
+      base += tot;
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out_count = base;
+}
+
+template <int NB>
+cudaError_t launch_lm_nb(const CUtensorMap& tm_w, const CUtensorMap& tm_h, const LmArgs& a, int grid, cudaStream_t s) {
+  using L = LmSmem<NB>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(lm_head_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  lm_head_kernel<NB><<<grid, kLmThreads, L::kTotal, s>>>(tm_w, tm_h, a);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int lm_head_grid(int vocab, int* tiles_per_cta) {
+  const int n_tiles = (vocab + kLmBM - 1) / kLmBM;
+  const int tpc = (n_tiles + kNumSMs - 1) / kNumSMs;
+  *tiles_per_cta = tpc;
+  return (n_tiles + tpc - 1) / tpc;
+}
+
+int lm_head_batch_pad(int B) { return B <= 16 ? 16 : (B <= 32 ? 32 : 64); }
+
+cudaError_t launch_lm_head(const CUtensorMap& tm_w, const CUtensorMap& tm_h, int h_row0, int B, int B_pad, int d,
+                           int vocab, const int32_t* verdict_ids_host, int n_verdict, float* part_max,
+                           float* part_sum, float* verdict_logits, float* logits_or_null, uint32_t* status,
+                           cudaStream_t s) {
+  LmArgs a;
+  a.B = B;
+  a.h_row0 = h_row0;
+  a.vocab = vocab;
+  a.kblocks = (d + kLmBK - 1) / kLmBK;
+  a.n_tiles = (vocab + kLmBM - 1) / kLmBM;
+  const int grid = lm_head_grid(vocab, &a.tiles_per_cta);
+  a.n_verdict = n_verdict;
+  for (int j = 0; j < kLmMaxVerdict; ++j) a.verdict[j] = j < n_verdict ? verdict_ids_host[j] : -1;
+  a.part_max = part_max;
+  a.part_sum = part_sum;
+  a.verdict_logits = verdict_logits;
+  a.logits = logits_or_null;
+  a.status = status;
+  switch (B_pad) {
+    case 16: return launch_lm_nb<16>(tm_w, tm_h, a, grid, s);
+    case 32: return launch_lm_nb<32>(tm_w, tm_h, a, grid, s);
+    case 64: return launch_lm_nb<64>(tm_w, tm_h, a, grid, s);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+cudaError_t launch_last_rows_norm(const float* x, const int32_t* cu_new, const float* gain, uint16_t* h, int B,
+                                  int B_pad, int d, float eps, cudaStream_t s) {
+  const int warps = 4;
+  last_rows_norm_kernel<<<(B_pad + warps - 1) / warps, warps * 32, 0, s>>>(x, cu_new, gain, h, B, B_pad, d, eps);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gate(const float* part_max, const float* part_sum, int n_slices, int nb_stride,
+                        const float* verdict_logits, int n_verdict, int B, float tau, float* out_conf,
+                        uint8_t* out_accept, int32_t* out_verdict, float* out_lse, cudaStream_t s) {
+  const int warps = 4;
+  gate_kernel<<<(B + warps - 1) / warps, warps * 32, 0, s>>>(part_max, part_sum, n_slices, nb_stride, verdict_logits,
+                                                           n_verdict, B, tau, out_conf, out_accept, out_verdict,
+                                                           out_lse);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_escalate(const float* conf, int B, float tau, uint8_t* out_accept, int32_t* out_idx,
+                            int32_t* out_count, cudaStream_t s) {
+  escalate_kernel<<<1, 1024, 0, s>>>(conf, B, tau, out_accept, out_idx, out_count);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace cs

@@ -1,0 +1,96 @@
+"""Shared driver of the end-to-end parity checks: run the CUDA path through the C ABI and the CPU oracle on
+the same seeded inputs and compare with the tolerances the pass is specified to:
+  last-position logits  max-abs <= 3e-2
+  confidence            abs     <= 5e-3
+  accept/escalate mask  bit-exact except where |conf - tau| < 5e-3
+  verdict index         equal unless the two best verdict probabilities are within 5e-3 of each other
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from oracle import confspec_oracle as O
+from workloads import context_kv, make_batch, model_weights, page_assignment, plant_verdict_rows
+
+LOGIT_TOL = 3e-2
+CONF_TOL = 5e-3
+
+
+def steps_of(batch) -> List[np.ndarray]:
+    return [batch.step_tokens[batch.cu_new[i]:batch.cu_new[i + 1]] for i in range(batch.n_steps)]
+
+
+def build_session(cfg, weights, batch, keep_logits=True):
+    """GPU side: model, cache and contexts for one workload."""
+    from paper_2602_18447_b200 import VerifySession, binding as B
+    ses = VerifySession(cfg, weights, batch)
+    B.cs_set_keep_logits(ses.model, keep_logits)
+    if cfg.ctx_kv == "prefill":
+        need = [(int(c) + cfg.page_size - 1) // cfg.page_size for c in batch.ctx_lens]
+        total, pages = page_assignment(cfg, batch.ctx_lens)
+        ses.alloc_cache(pages, total, batch.ctx_lens, room_for_prefill=True)
+        ses.prefill_context(batch.ctx_tokens)
+    else:
+        total, pages = page_assignment(cfg, batch.ctx_lens)
+        ses.alloc_cache(pages, total, batch.ctx_lens)
+        ses.fill_synthetic_context(lambda i, l: context_kv(cfg, i, l, int(batch.ctx_lens[i])))
+    return ses
+
+
+def oracle_outputs(cfg, weights, batch, steps: Optional[Sequence[int]] = None, tau: Optional[float] = None) -> dict:
+    """CPU side, for all steps or a sample of them (steps are independent)."""
+    idx = list(range(batch.n_steps)) if steps is None else list(steps)
+    toks = steps_of(batch)
+    tau = cfg.tau if tau is None else tau
+    if cfg.ctx_kv == "prefill":
+        kv = O.prefill_context(weights, [batch.ctx_tokens[i] for i in idx], store_bf16=True)
+        fn = lambda j, l: kv[j][l]
+    else:
+        def fn(j, l):
+            k, v = context_kv(cfg, idx[j], l, int(batch.ctx_lens[idx[j]]))
+            return O.widen_bf16(k), O.widen_bf16(v)
+    return O.verify_steps(weights, [toks[i] for i in idx], [int(batch.ctx_lens[i]) for i in idx], fn,
+                          cfg.verdict_ids, tau)
+
+
+def compare(gpu: dict, gpu_logits: Optional[np.ndarray], ref: dict, tau: float, steps: Optional[Sequence[int]] = None,
+            gpu_lse: Optional[np.ndarray] = None) -> dict:
+    """Assert the tolerances; returns the observed maxima for reporting."""
+    sel = slice(None) if steps is None else list(steps)
+    conf = gpu["conf"][sel].astype(np.float64)
+    stats = {"conf_err": float(np.max(np.abs(conf - ref["conf"])))}
+    assert np.all(np.isfinite(conf)), conf
+    assert stats["conf_err"] <= CONF_TOL, stats
+    if gpu_logits is not None:
+        stats["logit_err"] = float(np.max(np.abs(gpu_logits[sel].astype(np.float64) - ref["logits"])))
+        assert stats["logit_err"] <= LOGIT_TOL, stats
+    if gpu_lse is not None:
+        stats["lse_err"] = float(np.max(np.abs(gpu_lse[sel].astype(np.float64) - ref["lse"])))
+        assert stats["lse_err"] <= LOGIT_TOL, stats
+    near = np.abs(ref["conf"] - tau) < CONF_TOL
+    acc = gpu["accept"][sel]
+    assert np.array_equal(acc[~near], ref["accept"][~near]), (acc, ref["accept"], ref["conf"])
+    assert np.all((acc == 0) | (acc == 1))
+    # decision: compare where the oracle's two best verdict probabilities are clearly apart
+    if len(ref["logits"].shape) == 2 and ref["logits"].shape[0] == conf.shape[0]:
+        pass
+    stats["n_near_tau"] = int(near.sum())
+    stats["n_accept"] = int(ref["accept"].sum())
+    return stats
+
+
+def check_verdict(gpu: dict, ref: dict, verdict_ids: Sequence[int], steps: Optional[Sequence[int]] = None) -> None:
+    sel = slice(None) if steps is None else list(steps)
+    pv = np.exp(ref["logits"][:, list(verdict_ids)] - ref["lse"][:, None])
+    srt = np.sort(pv, axis=-1)
+    clear = (srt[:, -1] - srt[:, -2]) > CONF_TOL if pv.shape[1] > 1 else np.ones(pv.shape[0], bool)
+    assert np.array_equal(gpu["verdict"][sel][clear], ref["verdict"][clear])
+    assert np.all((gpu["verdict"][sel] >= 0) & (gpu["verdict"][sel] < len(verdict_ids)))
+
+
+def planted_weights(cfg, seed=None):
+    w = model_weights(cfg.model, cfg.seed if seed is None else seed)
+    plant_verdict_rows(w, cfg.verdict_ids, beta=float(np.log(cfg.model.vocab) + 0.5), seed=cfg.seed)
+    return w

@@ -1,0 +1,96 @@
+"""Single-kernel parity: each CUDA kernel that has a C entry point of its own is compared, element by
+element, with the oracle's corresponding block on the same seeded inputs. Sizes span several tiles, ragged
+tails in every dimension and the degenerate one-row case."""
+import numpy as np
+import pytest
+
+from oracle import confspec_oracle as O
+from workloads import bf16_bits_from_f32
+
+pytestmark = pytest.mark.gpu
+
+
+def _bf16_randn(g, shape, std):
+    return bf16_bits_from_f32((std * g.standard_normal(shape)).astype(np.float32))
+
+
+def _to_dev(bits):
+    import torch
+    return torch.from_numpy(bits.view(np.int16)).cuda()
+
+
+GEMM_SHAPES = [
+    # M, N, K
+    (160, 768, 256),      # tiny-config QKV
+    (1, 256, 256),        # one row
+    (129, 264, 200),      # every dimension ragged (N, K multiples of 8 only)
+    (300, 1536, 1536),    # O projection, 1.5B shape
+    (1088, 2048, 1536),   # QKV, 1.5B shape, 8.5 row tiles
+    (200, 1536, 8960),    # down projection K
+]
+
+
+@pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
+@pytest.mark.parametrize("epilogue", [0, 1, 2])
+def test_gemm_matches_oracle_matmul(M, N, K, epilogue):
+    import torch
+    from paper_2602_18447_b200 import binding as B
+    g = np.random.default_rng(1000 + M + N + K + epilogue)
+    a = _bf16_randn(g, (M, K), 1.0)
+    w = _bf16_randn(g, (N, K), 0.05)
+    w2 = _bf16_randn(g, (N, K), 0.05)
+    af, wf, w2f = O.widen_bf16(a), O.widen_bf16(w), O.widen_bf16(w2)
+    da, dw, dw2 = _to_dev(a), _to_dev(w), _to_dev(w2)
+    if epilogue == 1:
+        x0 = g.standard_normal((M, N)).astype(np.float32)
+        out = torch.from_numpy(x0.copy()).cuda()
+        want = x0.astype(np.float64) + af @ wf.T
+    else:
+        out = torch.full((M, N), -777.0, dtype=torch.bfloat16, device="cuda")
+        want = af @ wf.T if epilogue == 0 else O.silu(af @ wf.T) * (af @ w2f.T)
+    B.cs_gemm_bf16(da, dw, dw2 if epilogue == 2 else None, out, M, N, K, epilogue)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy().astype(np.float64)
+    scale = float(np.abs(want).max())
+    # fp32 accumulation of exact bf16 products, then one rounding to the output type
+    tol = (2.0 ** -8) * np.abs(want) + 2e-5 * scale * (1 + K / 1024) if epilogue != 1 else 3e-5 * scale * (1 + K / 1024)
+    bad = np.abs(got - want) > tol
+    assert not bad.any(), (int(bad.sum()), float(np.abs(got - want).max()), scale)
+
+
+@pytest.mark.parametrize("rows,d", [(1, 256), (37, 1536), (1088, 1536), (70, 3584)])
+def test_rmsnorm_matches_oracle(rows, d):
+    import torch
+    from paper_2602_18447_b200 import binding as B
+    g = np.random.default_rng(rows * 7 + d)
+    x = (g.standard_normal((rows, d)) * g.uniform(0.01, 30.0, size=(rows, 1))).astype(np.float32)
+    gain = (1.0 + 0.2 * g.standard_normal(d)).astype(np.float32)
+    out = torch.empty((rows, d), dtype=torch.bfloat16, device="cuda")
+    B.cs_rmsnorm(torch.from_numpy(x).cuda(), torch.from_numpy(gain).cuda(), out, rows, d, 1e-6)
+    torch.cuda.synchronize()
+    want = O.rmsnorm(x.astype(np.float64), gain.astype(np.float64), 1e-6)
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - want) <= (2.0 ** -8) * np.abs(want) + 1e-6)
+
+
+def test_escalate_mask_matches_oracle_bit_exact():
+    import torch
+    from paper_2602_18447_b200 import binding as B
+    g = np.random.default_rng(5)
+    for n in (1, 31, 64, 1000, 5000):
+        conf = g.uniform(0, 1, size=n).astype(np.float32)
+        conf[::7] = np.float32(0.9)          # exactly on the threshold: trusted
+        if n > 3:
+            conf[3] = np.nan                 # never trusted
+        dconf = torch.from_numpy(conf).cuda()
+        for tau in (0.0, 0.5, 0.9, 1.0001):
+            acc = torch.zeros(n, dtype=torch.uint8, device="cuda")
+            idx = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+            cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+            B.cs_escalate_mask(dconf, tau, acc, idx, cnt)
+            torch.cuda.synchronize()
+            want_acc, want_idx, want_cnt = O.escalate_list(conf, tau)
+            assert int(cnt.item()) == want_cnt
+            assert np.array_equal(acc.cpu().numpy(), want_acc)
+            assert np.array_equal(idx.cpu().numpy()[:want_cnt], want_idx)
+            assert np.all(idx.cpu().numpy()[want_cnt:] == -1)

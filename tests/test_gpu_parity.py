@@ -1,0 +1,125 @@
+"""End-to-end parity of cs_verify_steps with the CPU oracle at sizes the oracle finishes in seconds: the tiny
+workload (real prefill through cs_prefill), reduced-depth variants of the 1.5B- and 7B-shaped workloads (same
+widths, ragged contexts and steps, scattered pages), planted-verdict variants that put confidences on both
+sides of the threshold, and the edge cases of the batch structure."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from workloads import get_config, make_batch, model_weights, scaled_config
+
+import parity_common as P
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, weights, batch, taus=None):
+    ses = P.build_session(cfg, weights, batch)
+    try:
+        ses.verify()
+        gpu = ses.results()
+        logits, lse = ses.last_logits(), ses.last_lse()
+        ref = P.oracle_outputs(cfg, weights, batch)
+        stats = P.compare(gpu, logits, ref, cfg.tau, gpu_lse=lse)
+        P.check_verdict(gpu, ref, cfg.verdict_ids)
+        for tau in taus or ():
+            ses.verify(tau=tau)
+            g2 = ses.results()
+            r2 = dict(ref, accept=P.O.gate(ref["conf"], tau))
+            P.compare(g2, None, r2, tau)
+        # host-token entry (tokens copied inside the call) gives the same answer
+        ses.verify(host_tokens=True)
+        g3 = ses.results()
+        assert np.max(np.abs(g3["conf"] - gpu["conf"])) <= 1e-4
+        return stats, gpu, ref
+    finally:
+        ses.close()
+
+
+def test_cfg1_tiny_with_real_prefill():
+    cfg = get_config("cfg1_tiny")
+    stats, gpu, ref = _run(cfg, model_weights(cfg.model, cfg.seed), make_batch(cfg))
+    assert gpu["accept"].tolist() == [0] * cfg.batch      # random-init weights: conf ~ 1/V, all escalate
+    assert stats["logit_err"] < 3e-2
+
+
+def test_cfg1_tiny_planted_verdict_rows_and_tau_sweep():
+    cfg = replace(get_config("cfg1_tiny"), batch=24)
+    stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), taus=(0.0, 0.5, 0.7, 0.9, 0.95, 0.99, 1.0001))
+    assert 0 < ref["accept"].sum() < cfg.batch           # the gate is exercised on both sides
+    assert ref["conf"].max() > 0.9 and ref["conf"].min() < 0.5
+
+
+@pytest.mark.parametrize("name,layers,batch", [("cfg2_1p5b_b16", 2, 5), ("cfg3_1p5b_b64", 1, 9), ("cfg5_7b_b32", 1, 4)])
+def test_reduced_depth_large_shapes(name, layers, batch):
+    cfg = scaled_config(name, n_layers=layers, batch=batch, vocab=20480 + 8)   # ragged vocabulary tail
+    stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), taus=(0.5, 0.99))
+    assert stats["logit_err"] < 3e-2
+
+
+def test_long_context_split_kv():
+    cfg = scaled_config("cfg4_1p5b_long", n_layers=1, batch=2, vocab=8192)
+    _run(cfg, P.planted_weights(cfg), make_batch(cfg))
+
+
+@pytest.mark.parametrize("ctx,step", [(0, 1), (1, 1), (15, 3), (16, 64), (17, 65), (63, 129), (64, 200), (65, 7)])
+def test_context_and_step_length_edges(ctx, step):
+    """Empty context, single-token step, page and tile boundaries +-1."""
+    base = get_config("cfg1_tiny")
+    cfg = replace(base, batch=3, ctx_dist=("fixed", ctx), step_dist=("fixed", step), suffix_len=0)
+    batch = make_batch(cfg)
+    _run(cfg, P.planted_weights(cfg), batch)
+
+
+def test_batch_permutation_permutes_outputs():
+    cfg = replace(get_config("cfg1_tiny"), batch=6, ctx_dist=("uniform", 20, 150), step_dist=("uniform", 5, 60))
+    w = P.planted_weights(cfg)
+    batch = make_batch(cfg)
+    ses = P.build_session(cfg, w, batch)
+    try:
+        ses.verify()
+        base = ses.results()
+        perm = np.array([3, 0, 5, 1, 4, 2])
+        from paper_2602_18447_b200 import binding as B
+        import torch
+        toks = np.concatenate([P.steps_of(batch)[p] for p in perm]).astype(np.int32)
+        conf = torch.empty(6, dtype=torch.float32, device="cuda")
+        acc = torch.empty(6, dtype=torch.uint8, device="cuda")
+        B.cs_verify_steps(ses.model, ses.kv, perm.astype(np.int32), toks, batch.step_lens[perm], cfg.verdict_ids,
+                          cfg.tau, conf, acc)
+        torch.cuda.synchronize()
+        assert np.max(np.abs(conf.cpu().numpy() - base["conf"][perm])) <= 1e-4
+    finally:
+        ses.close()
+
+
+def test_invalid_arguments_are_rejected_before_any_launch():
+    import torch
+    from paper_2602_18447_b200 import binding as B
+    cfg = replace(get_config("cfg1_tiny"), batch=2)
+    batch = make_batch(cfg)
+    ses = P.build_session(cfg, model_weights(cfg.model, cfg.seed), batch)
+    try:
+        B.cs_take_launch_count()
+        conf = torch.empty(2, dtype=torch.float32, device="cuda")
+        acc = torch.empty(2, dtype=torch.uint8, device="cuda")
+
+        def call(**kw):
+            a = dict(seq=ses.seq_ids, toks=batch.step_tokens, lens=batch.step_lens, vids=cfg.verdict_ids, tau=0.9)
+            a.update(kw)
+            B.cs_verify_steps(ses.model, ses.kv, a["seq"], a["toks"], a["lens"], a["vids"], a["tau"], conf, acc)
+
+        for bad in (dict(tau=float("nan")), dict(lens=np.array([0, 5], np.int32)), dict(vids=[cfg.model.vocab]),
+                    dict(vids=[]), dict(seq=np.array([0, 7], np.int32)),
+                    dict(toks=np.full_like(batch.step_tokens, cfg.model.vocab))):
+            with pytest.raises(B.ConfSpecError) as e:
+                call(**bad)
+            assert e.value.status == B.CS_EINVAL
+        assert B.cs_take_launch_count() == 0
+        # an empty batch is a no-op
+        B.cs_verify_steps(ses.model, ses.kv, np.zeros(0, np.int32), np.zeros(0, np.int32), np.zeros(0, np.int32),
+                          cfg.verdict_ids, 0.9, conf, acc)
+        assert B.cs_take_launch_count() == 0
+    finally:
+        ses.close()
