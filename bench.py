@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Throughput of the batched draft-verification pass.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one cs_verify_steps call over the whole batch of the workload (every kernel of the pass).
+Prints ONE JSON line. With --gpus N > 1 (launched by torch.distributed.run) every rank runs an independent
+replica on its own seeded batch: the pass has no exchange step, so there is no collective on the data path.
+`--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from workloads import context_kv, get_config, make_batch, model_weights, page_assignment  # noqa: E402
+
+METRIC = "verified_steps_per_s"
+UNIT = "steps/s"
+DEFAULT_WORKLOAD = "cfg2_1p5b_b16"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic work of the pass (per call)
+# ------------------------------------------------------------------------------------------------
+def work_counts(cfg, batch) -> dict:
+    m = cfg.model
+    T = int(batch.n_tokens)
+    n = batch.step_lens.astype(np.float64)
+    c = batch.ctx_lens.astype(np.float64)
+    attn_flops_layer = float(np.sum(4.0 * m.n_q_heads * m.head_dim * (n * c + n * (n + 1) / 2)))
+    kv_row = 2 * m.n_kv_heads * m.head_dim * 2                       # bytes of K+V per token per layer
+    attn_bytes_layer = float(np.sum(c) * kv_row + T * (m.q_dim + 2 * m.kv_dim + m.q_dim) * 2)
+    return {
+        "T": T,
+        "gemm_qkv_flops": 2.0 * T * (m.q_dim + 2 * m.kv_dim) * m.d_model,
+        "gemm_o_flops": 2.0 * T * m.d_model * m.q_dim,
+        "gemm_gateup_flops": 2.0 * T * (2 * m.d_ffn) * m.d_model,
+        "gemm_down_flops": 2.0 * T * m.d_model * m.d_ffn,
+        "attention_flops": attn_flops_layer,
+        "attention_bytes": attn_bytes_layer,
+        "lm_head_bytes": 2.0 * m.vocab * m.d_model + batch.n_steps * m.d_model * 2,
+        "lm_head_flops": 2.0 * batch.n_steps * m.vocab * m.d_model,
+    }
+
+
+# ------------------------------------------------------------------------------------------------
+# clock sampling during the timed region
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_uuid: str):
+        self.rows = []
+        self.proc = None
+        self.uuid = gpu_uuid
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", self.uuid], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self, t0: float, t1: float) -> dict:
+        sm, mx, reasons = [], [], set()
+        for ts, line in self.rows:
+            if ts < t0 or ts > t1 + 0.2:
+                continue
+            p = [x.strip() for x in line.split(",")]
+            if len(p) < 7:
+                continue
+            try:
+                sm.append(float(p[0]))
+                mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle leg (bounded sample)
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_run(cfg, weights, batch, sample_steps):
+    """One oracle pass over `sample_steps` of the batch; returns seconds."""
+    from oracle import confspec_oracle as O
+    toks = [batch.step_tokens[batch.cu_new[i]:batch.cu_new[i + 1]] for i in sample_steps]
+
+    def fn(j, l):
+        i = sample_steps[j]
+        k, v = context_kv(cfg, i, l, int(batch.ctx_lens[i]))
+        return O.widen_bf16(k), O.widen_bf16(v)
+
+    t = time.perf_counter()
+    if cfg.ctx_kv == "prefill":
+        kv = O.prefill_context(weights, [batch.ctx_tokens[i] for i in sample_steps], store_bf16=True)
+        fn = lambda j, l: kv[j][l]  # noqa: E731
+    O.verify_steps(weights, toks, [int(batch.ctx_lens[i]) for i in sample_steps], fn, cfg.verdict_ids, cfg.tau)
+    return time.perf_counter() - t
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return int(max(n)) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    weights = model_weights(cfg.model, cfg.seed)
+    batch = make_batch(cfg)
+    sample = list(range(min(2, batch.n_steps)))
+    for _ in range(args.warmup):
+        oracle_sample_run(cfg, weights, batch, sample[:1])
+    t = 0.0
+    for _ in range(args.steps):
+        t += oracle_sample_run(cfg, weights, batch, sample)
+    value = len(sample) * args.steps / t
+    tok = float(sum(int(batch.step_lens[i]) for i in sample)) * args.steps / t
+    desc = f"steps {sample} of the {batch.n_steps}-step batch per pass, context K/V generation included"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "tokens_per_s": tok,
+        "config": {"workload": cfg.name, "model": cfg.model.name, "batch": cfg.batch, "sampled_steps": len(sample)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA path
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_18447_b200 import VerifySession, binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the pass has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    weights = model_weights(cfg.model, cfg.seed)
+    batch = make_batch(cfg, seed=cfg.seed + 7919 * rank)       # each replica verifies its own batch
+    ses = VerifySession(cfg, weights, batch, device=f"cuda:{local}")
+    total, pages = page_assignment(cfg, batch.ctx_lens)
+    if cfg.ctx_kv == "prefill":
+        ses.alloc_cache(pages, total, batch.ctx_lens, room_for_prefill=True)
+        ses.prefill_context(batch.ctx_tokens)
+    else:
+        ses.alloc_cache(pages, total, batch.ctx_lens)
+        ses.fill_synthetic_context(lambda i, l: context_kv(cfg, i, l, int(batch.ctx_lens[i])))
+    B.cs_reserve(ses.model, batch.n_steps, batch.n_tokens)
+    stream = torch.cuda.current_stream()
+    K, W = args.steps, max(3, args.warmup)
+    counts = work_counts(cfg, batch)
+
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", ""))
+    sampler.start()
+    for _ in range(W):
+        ses.verify()
+    torch.cuda.synchronize()
+
+    # ---- device-resident throughput -------------------------------------------------------------
+    B.cs_take_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(K):
+        ses.verify()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    barrier()
+    launches = B.cs_take_launch_count()
+    ms = ev0.elapsed_time(ev1)
+    B.cs_last_status(ses.model)
+
+    # ---- end to end: host tokens in, results read back on the host, every step ---------------------
+    conf_host = torch.empty(batch.n_steps, dtype=torch.float32).pin_memory()
+    acc_host = torch.empty(batch.n_steps, dtype=torch.uint8).pin_memory()
+    for _ in range(2):
+        ses.verify(host_tokens=True)
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(K):
+        ses.verify(host_tokens=True)
+        conf_host.copy_(ses.out_conf, non_blocking=True)
+        acc_host.copy_(ses.out_accept, non_blocking=True)
+        stream.synchronize()                      # the caller reads the mask before its next step
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+
+    # ---- per-kernel durations (events around every launch; same workload, same process) -------------
+    B.cs_profile(ses.model, True)
+    for _ in range(K):
+        ses.verify()
+    torch.cuda.synchronize()
+    prof = B.cs_profile_read(ses.model)
+    B.cs_profile(ses.model, False)
+    sampler.stop()
+    clocks = sampler.summary(t_wall0, t_wall1)
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+        nb = torch.tensor([batch.n_steps, batch.n_tokens], dtype=torch.float64, device="cuda")
+        dist.all_reduce(nb, op=dist.ReduceOp.SUM)
+        all_steps, all_tokens = float(nb[0]), float(nb[1])
+    else:
+        all_steps, all_tokens = float(batch.n_steps), float(batch.n_tokens)
+
+    peaks, peak_kind = load_peaks()
+    tensor_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))   # fp16 and bf16 share the peak
+    hbm_peak = float(peaks["hbm_gbs"])
+
+    def per_launch_ms(name):
+        t_ms, n = prof[name]
+        return t_ms / n if n else float("nan")
+
+    L = cfg.model.n_layers
+    gu_ms = per_launch_ms("gemm_gateup")
+    gu_tf = counts["gemm_gateup_flops"] / (gu_ms * 1e-3) / 1e12
+    kernels = {}
+    for name, flops in (("gemm_qkv", counts["gemm_qkv_flops"]), ("gemm_o", counts["gemm_o_flops"]),
+                        ("gemm_gateup", counts["gemm_gateup_flops"]), ("gemm_down", counts["gemm_down_flops"])):
+        t_ms = per_launch_ms(name)
+        kernels[name] = {"ms_per_launch": t_ms, "tflops": flops / (t_ms * 1e-3) / 1e12,
+                         "frac_tensor": flops / (t_ms * 1e-3) / 1e12 / tensor_peak}
+    a_ms = per_launch_ms("attention")
+    kernels["attention"] = {"ms_per_launch": a_ms, "tflops": counts["attention_flops"] / (a_ms * 1e-3) / 1e12,
+                            "frac_tensor": counts["attention_flops"] / (a_ms * 1e-3) / 1e12 / tensor_peak,
+                            "gbs": counts["attention_bytes"] / (a_ms * 1e-3) / 1e9,
+                            "frac_hbm": counts["attention_bytes"] / (a_ms * 1e-3) / 1e9 / hbm_peak}
+    l_ms = per_launch_ms("lm_head")
+    kernels["lm_head"] = {"ms_per_launch": l_ms, "gbs": counts["lm_head_bytes"] / (l_ms * 1e-3) / 1e9,
+                          "frac_hbm": counts["lm_head_bytes"] / (l_ms * 1e-3) / 1e9 / hbm_peak}
+    prof_total = sum(v[0] for v in prof.values())
+    shares = {k: (v[0] / prof_total if prof_total else 0.0) for k, v in prof.items()}
+
+    out = {
+        "metric": METRIC, "value": all_steps * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16", "data": "synthetic",
+        "tokens_per_s": all_tokens * K / (ms * 1e-3),
+        "config": {"workload": cfg.name, "model": cfg.model.name, "batch": cfg.batch, "new_tokens": counts["T"],
+                   "ctx_tokens": int(batch.ctx_lens.sum()), "tau": cfg.tau, "page_size": cfg.page_size,
+                   "l2": "inputs larger than L2 (3.1 GB of weights streamed every step)",
+                   "replicas": world},
+        "clocks": clocks,
+        "e2e": {"value": all_steps * K / (ms_e2e * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": int(batch.n_tokens * 4 + (6 * batch.n_steps + 2 * batch.n_tokens) * 4),
+                "d2h_bytes_per_step": int(batch.n_steps * 5), "ms_per_step": ms_e2e / K},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "gemm_f16_kernel<256, SwiGLU> (gate/up projection)", "bound": "tensor",
+                     "achieved": gu_tf, "peak": tensor_peak, "unit": "TFLOP/s", "frac": gu_tf / tensor_peak,
+                     "peak_kind": f"{peak_kind} bf16 sustained (fp16 has the same nominal peak)",
+                     "traffic": None, "ms_per_launch": gu_ms, "launches_timed": prof["gemm_gateup"][1]},
+        "kernels": kernels,
+        "time_shares": shares,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample = list(range(min(3, batch.n_steps)))
+        t = oracle_sample_run(cfg, weights, batch, sample)
+        out["cpu_baseline"] = {"value": len(sample) / t, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                               "sample": f"one oracle pass over steps {sample} of the {batch.n_steps}-step batch "
+                                         f"({t:.1f} s, context K/V generation included)"}
+    ses.close()
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = get_config(args.workload)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

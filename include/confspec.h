@@ -74,7 +74,10 @@ const char* cs_last_cuda_error(void);
 /*
  * cs_model_load — copy a verifier model (the M_D, or M_T for escalated steps, of Algorithm 1) into
  * library-owned device memory and prepare everything that does not depend on a batch (fused QKV matrix,
- * TMA descriptors, rotary frequencies).
+ * TMA descriptors, rotary frequencies). The projection and LM-head matrices are re-encoded from bf16 to fp16
+ * on the device (exact for magnitudes in [2^-14, 65504], absolute error <= 2^-25 below): the tensor cores take
+ * both operands in one 16-bit format, and the activations are kept in fp16, whose rounding error is 8x smaller
+ * than bf16's. Activations beyond the fp16 range (|v| > 65504) are not supported.
  *   desc               host. Geometry.
  *   tensors            host struct; the tensor pointers inside are host pointers when
  *                      tensors_on_device == 0, device pointers otherwise. The caller keeps ownership and
@@ -191,15 +194,26 @@ int cs_last_status(cs_model* model, void* stream);
  * Per-stage entry points. They run single kernels of the pass on caller-provided device buffers so that
  * each can be checked against the oracle's corresponding block, and timed, in isolation.
  */
-/* out[M,N] (+)= a[M,K] * w[N,K]^T on the tcgen05 tensor cores. a, w bf16 row-major.
- *   epilogue 0: out bf16 [M,N] = result.
+/* out[M,N] (+)= a[M,K] * w[N,K]^T on the tcgen05 tensor cores. a, w fp16 row-major (device), fp32 accumulate.
+ *   epilogue 0: out fp16 [M,N] = result.
  *   epilogue 1: out fp32 [M,N] += result (atomic adds; split along K over the SMs).
- *   epilogue 2: w2 is a second [N,K] matrix; out bf16 [M,N] = silu(a*w^T) * (a*w2^T).
+ *   epilogue 2: w2 is a second [N,K] matrix; out fp16 [M,N] = silu(a*w^T) * (a*w2^T).
  * K and N multiples of 8. Asynchronous on `stream`. */
-int cs_gemm_bf16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* out,
+int cs_gemm_f16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* out,
                  int M, int N, int K, int epilogue, void* stream);
-/* out bf16 [rows, d] = RMSNorm(x fp32 [rows, d]; gain fp32 [d], eps). */
+/* out fp16 [rows, d] = RMSNorm(x fp32 [rows, d]; gain fp32 [d], eps). */
 int cs_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps, void* stream);
+/*
+ * Per-kernel-class timing of the pass. cs_profile(model, 1) makes cs_verify_steps / cs_prefill record a pair
+ * of CUDA events around each kernel launch (on the call's stream); cs_profile_read waits for the recorded
+ * events, adds the elapsed milliseconds and the number of timed launches per class into ms_out / calls_out
+ * (host arrays of n_classes >= CS_PROF_CLASSES entries) and clears the record. Classes, in order: embedding,
+ * RMSNorm, QKV GEMM, rotary, attention (+ merge), O GEMM, gate/up GEMM (SwiGLU), down GEMM, LM head, gate,
+ * other. The events cost a little host and device time, so throughput is measured with profiling off.
+ */
+#define CS_PROF_CLASSES 11
+int cs_profile(cs_model* model, int enable);
+int cs_profile_read(cs_model* model, float* ms_out, int32_t* calls_out, int n_classes);
 /* Number of kernels the library has launched on this host thread since the last call of this function. */
 int64_t cs_take_launch_count(void);
 

@@ -17,8 +17,11 @@ EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_reserve",
     "cs_kv_alloc", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
     "cs_verify_steps", "cs_escalate_mask", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
-    "cs_last_status", "cs_gemm_bf16", "cs_rmsnorm", "cs_take_launch_count",
+    "cs_last_status", "cs_gemm_f16", "cs_rmsnorm", "cs_take_launch_count", "cs_profile", "cs_profile_read",
 ]
+
+PROF_CLASSES = ["embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gateup", "gemm_down",
+                "lm_head", "gate", "other"]
 
 
 class ConfSpecError(RuntimeError):
@@ -75,9 +78,11 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_get_last_logits": (C.c_int, [vp, vp, i32, vp]),
         "cs_get_last_lse": (C.c_int, [vp, vp, i32, vp]),
         "cs_last_status": (C.c_int, [vp, vp]),
-        "cs_gemm_bf16": (C.c_int, [vp, vp, vp, vp, i32, i32, i32, i32, vp]),
+        "cs_gemm_f16": (C.c_int, [vp, vp, vp, vp, i32, i32, i32, i32, vp]),
         "cs_rmsnorm": (C.c_int, [vp, vp, vp, i32, i32, f32, vp]),
         "cs_take_launch_count": (C.c_int64, []),
+        "cs_profile": (C.c_int, [vp, i32]),
+        "cs_profile_read": (C.c_int, [vp, vp, vp, i32]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)   # AttributeError if the symbol is not exported
@@ -242,11 +247,24 @@ def cs_last_status(model: int, stream=None) -> None:
     _check(load_library().cs_last_status(model, _stream_ptr(stream)), "cs_last_status")
 
 
-def cs_gemm_bf16(a, w, w2, out, M: int, N: int, K: int, epilogue: int, stream=None) -> None:
-    _check(load_library().cs_gemm_bf16(_dev_ptr(a), _dev_ptr(w), _dev_ptr(w2), _dev_ptr(out), M, N, K, epilogue,
-                                       _stream_ptr(stream)), "cs_gemm_bf16")
+def cs_gemm_f16(a, w, w2, out, M: int, N: int, K: int, epilogue: int, stream=None) -> None:
+    _check(load_library().cs_gemm_f16(_dev_ptr(a), _dev_ptr(w), _dev_ptr(w2), _dev_ptr(out), M, N, K, epilogue,
+                                       _stream_ptr(stream)), "cs_gemm_f16")
 
 
 def cs_rmsnorm(x, gain, out, rows: int, d: int, eps: float, stream=None) -> None:
     _check(load_library().cs_rmsnorm(_dev_ptr(x), _dev_ptr(gain), _dev_ptr(out), rows, d, float(eps),
                                      _stream_ptr(stream)), "cs_rmsnorm")
+
+
+def cs_profile(model: int, enable: bool) -> None:
+    _check(load_library().cs_profile(model, 1 if enable else 0), "cs_profile")
+
+
+def cs_profile_read(model: int) -> dict:
+    """{class name: (milliseconds, timed launches)} since profiling was enabled or last read."""
+    n = len(PROF_CLASSES)
+    ms = np.zeros(n, dtype=np.float32)
+    calls = np.zeros(n, dtype=np.int32)
+    _check(load_library().cs_profile_read(model, _np_ptr(ms), _np_ptr(calls), n), "cs_profile_read")
+    return {name: (float(ms[i]), int(calls[i])) for i, name in enumerate(PROF_CLASSES)}

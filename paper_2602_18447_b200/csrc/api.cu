@@ -62,6 +62,16 @@ struct DevBuf {
   }
 };
 
+// Optional per-kernel-class timing: a pair of events around every launch of the pass.
+enum ProfClass { kProfEmbed = 0, kProfNorm, kProfQkv, kProfRope, kProfAttn, kProfO, kProfGateUp, kProfDown,
+                 kProfLmHead, kProfGate, kProfOther, kProfClasses };
+struct Prof {
+  bool on = false;
+  std::vector<cudaEvent_t> pool;   // events, used in pairs
+  std::vector<int> cls;            // class of pair i
+  size_t used = 0;                 // pairs in use
+};
+
 struct Staging {
   int32_t* host[kStagingRing] = {nullptr, nullptr, nullptr, nullptr};
   size_t host_cap[kStagingRing] = {0, 0, 0, 0};
@@ -88,6 +98,7 @@ struct cs_model {
   Staging stg;
   bool keep_logits = false;
   int last_B = 0;
+  Prof prof;
 };
 
 struct cs_kv {
@@ -214,6 +225,33 @@ int dev_copy(cs_model* m, T** dst, const T* src, size_t n, bool src_dev) {
   return CS_OK;
 }
 
+void prof_begin(cs_model* m, int cls, cudaStream_t s) {
+  Prof& p = m->prof;
+  if (!p.on) return;
+  if (p.pool.size() < 2 * (p.used + 1)) {
+    cudaEvent_t a = nullptr, b = nullptr;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { p.on = false; return; }
+    p.pool.push_back(a);
+    p.pool.push_back(b);
+    p.cls.push_back(cls);
+  }
+  p.cls[p.used] = cls;
+  cudaEventRecord(p.pool[2 * p.used], s);
+}
+void prof_end(cs_model* m, cudaStream_t s) {
+  Prof& p = m->prof;
+  if (!p.on) return;
+  cudaEventRecord(p.pool[2 * p.used + 1], s);
+  ++p.used;
+}
+#define CS_STEP(cls, call)                                \
+  do {                                                    \
+    prof_begin(m, cls, s);                                \
+    cudaError_t e__ = (call);                             \
+    prof_end(m, s);                                       \
+    if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+  } while (0)
+
 // The forward over all layers for a staged batch. When `append_kv` is given the new K/V of every layer are
 // also written to that cache's pages.
 int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout& L, const int32_t* dev_meta,
@@ -238,13 +276,13 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   CUtensorMap tm_a, tm_o, tm_h, tm_qkv_attn;
   if (!make_gemm_operand_map(&tm_a, a, T, d.d_model) || !make_gemm_operand_map(&tm_o, attn_o, T, m->q_dim) ||
       !make_gemm_operand_map(&tm_h, hmlp, T, d.d_ffn) ||
-      !make_tensor_map_bf16(&tm_qkv_attn, qkv, T, m->n_qkv, kPageSize, 64, true)) {
+      !make_tensor_map_16b(&tm_qkv_attn, qkv, T, m->n_qkv, kPageSize, 64, true, false)) {
     g_cuda_error = "cuTensorMapEncodeTiled failed for an activation buffer";
     return CS_ECUDA;
   }
 
-  CS_CUDA(launch_embed(d_tok, m->embed, x, T, d.d_model, d.vocab, s));
-  CS_CUDA(launch_rope_table(d_pos, m->inv_freq, rope, T, d.head_dim / 2, s));
+  CS_STEP(kProfEmbed, launch_embed(d_tok, m->embed, x, T, d.d_model, d.vocab, s));
+  CS_STEP(kProfOther, launch_rope_table(d_pos, m->inv_freq, rope, T, d.head_dim / 2, s));
 
   AttnParams ap;
   ap.qkv = qkv;
@@ -266,23 +304,23 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
 
   for (int l = 0; l < d.n_layers; ++l) {
     const LayerDev& lw = m->layers[l];
-    CS_CUDA(launch_rmsnorm(x, lw.norm1, a, T, d.d_model, d.rms_eps, s));
-    CS_CUDA(gemm_bf16(tm_a, lw.tm_wqkv, nullptr, qkv, T, m->n_qkv, d.d_model, kEpiStoreBf16, m->status, s));
-    CS_CUDA(launch_rope_apply(qkv, rope, T, m->n_qkv, d.n_q_heads + d.n_kv_heads, d.head_dim, s));
+    CS_STEP(kProfNorm, launch_rmsnorm(x, lw.norm1, a, T, d.d_model, d.rms_eps, s));
+    CS_STEP(kProfQkv, gemm_f16(tm_a, lw.tm_wqkv, nullptr, qkv, T, m->n_qkv, d.d_model, kEpiStoreF16, m->status, s));
+    CS_STEP(kProfRope, launch_rope_apply(qkv, rope, T, m->n_qkv, d.n_q_heads + d.n_kv_heads, d.head_dim, s));
     ap.k_row_base = (2 * l) * plane_rows;
     ap.v_row_base = (2 * l + 1) * plane_rows;
-    CS_CUDA(launch_attention(ap, kv->tm_pool, tm_qkv_attn, d_items, L.n_items, d_merges, L.n_merges, s));
+    CS_STEP(kProfAttn, launch_attention(ap, kv->tm_pool, tm_qkv_attn, d_items, L.n_items, d_merges, L.n_merges, s));
     if (append_kv) {
-      CS_CUDA(launch_kv_scatter(qkv + m->q_dim, qkv + m->q_dim + m->kv_dim, m->n_qkv, d_tseq, d_pos, 0, 0,
+      CS_STEP(kProfOther, launch_kv_scatter(qkv + m->q_dim, qkv + m->q_dim + m->kv_dim, m->n_qkv, d_tseq, d_pos, 0, 0,
                                 append_kv->table_dev, append_kv->max_pages_per_seq,
                                 append_kv->pool + static_cast<size_t>(2 * l) * append_kv->plane_elems,
                                 append_kv->pool + static_cast<size_t>(2 * l + 1) * append_kv->plane_elems,
-                                d.n_kv_heads, d.head_dim, kPageSize, T, s));
+                                d.n_kv_heads, d.head_dim, kPageSize, T, 1, s));
     }
-    CS_CUDA(gemm_bf16(tm_o, lw.tm_wo, nullptr, x, T, d.d_model, m->q_dim, kEpiResidAdd, m->status, s));
-    CS_CUDA(launch_rmsnorm(x, lw.norm2, a, T, d.d_model, d.rms_eps, s));
-    CS_CUDA(gemm_bf16(tm_a, lw.tm_wg, &lw.tm_wu, hmlp, T, d.d_ffn, d.d_model, kEpiSwiGLU, m->status, s));
-    CS_CUDA(gemm_bf16(tm_h, lw.tm_wd, nullptr, x, T, d.d_model, d.d_ffn, kEpiResidAdd, m->status, s));
+    CS_STEP(kProfO, gemm_f16(tm_o, lw.tm_wo, nullptr, x, T, d.d_model, m->q_dim, kEpiResidAdd, m->status, s));
+    CS_STEP(kProfNorm, launch_rmsnorm(x, lw.norm2, a, T, d.d_model, d.rms_eps, s));
+    CS_STEP(kProfGateUp, gemm_f16(tm_a, lw.tm_wg, &lw.tm_wu, hmlp, T, d.d_ffn, d.d_model, kEpiSwiGLU, m->status, s));
+    CS_STEP(kProfDown, gemm_f16(tm_h, lw.tm_wd, nullptr, x, T, d.d_model, d.d_ffn, kEpiResidAdd, m->status, s));
   }
   return CS_OK;
 }
@@ -461,6 +499,14 @@ int cs_model_load(const cs_model_desc* desc, const cs_model_tensors* t, int on_d
     CS_TRY(dev_copy(m, &lw.wd, t->wd[l], dm * F, sd));
     CS_TRY(dev_copy(m, &lw.norm1, t->norm1[l], dm, sd));
     CS_TRY(dev_copy(m, &lw.norm2, t->norm2[l], dm, sd));
+    // The matrices arrive as bf16 and are kept as fp16 (same size; see launch_bf16_to_f16): the tensor cores
+    // take both operands in one 16-bit format and fp16 activations carry three more mantissa bits.
+    e = launch_bf16_to_f16(lw.wqkv, static_cast<size_t>(m->n_qkv) * dm, nullptr);
+    if (e == cudaSuccess) e = launch_bf16_to_f16(lw.wo, dm * m->q_dim, nullptr);
+    if (e == cudaSuccess) e = launch_bf16_to_f16(lw.wg, F * dm, nullptr);
+    if (e == cudaSuccess) e = launch_bf16_to_f16(lw.wu, F * dm, nullptr);
+    if (e == cudaSuccess) e = launch_bf16_to_f16(lw.wd, dm * F, nullptr);
+    if (e != cudaSuccess) { rc = cuda_fail(e, "bf16->fp16 weight conversion"); cs_model_free(m); return rc; }
     if (!make_gemm_operand_map(&lw.tm_wqkv, lw.wqkv, m->n_qkv, desc->d_model) ||
         !make_gemm_operand_map(&lw.tm_wo, lw.wo, desc->d_model, m->q_dim) ||
         !make_gemm_operand_map(&lw.tm_wg, lw.wg, desc->d_ffn, desc->d_model) ||
@@ -470,6 +516,10 @@ int cs_model_load(const cs_model_desc* desc, const cs_model_tensors* t, int on_d
       cs_model_free(m);
       return CS_ECUDA;
     }
+  }
+  {
+    cudaError_t e = launch_bf16_to_f16(m->lm_head, V * dm, nullptr);
+    if (e != cudaSuccess) { rc = cuda_fail(e, "bf16->fp16 weight conversion"); cs_model_free(m); return rc; }
   }
   if (!make_gemm_operand_map(&m->tm_lm, m->lm_head, desc->vocab, desc->d_model)) {
     g_cuda_error = "cuTensorMapEncodeTiled failed for the LM head";
@@ -504,6 +554,7 @@ int cs_model_free(cs_model* m) {
   DevBuf* bufs[] = {&m->x, &m->a, &m->qkv, &m->attn_o, &m->hmlp, &m->rope, &m->h_last, &m->lm_part, &m->vlogits,
                     &m->logits, &m->lse, &m->attn_part_o, &m->attn_part_ml, &m->stg.dev};
   for (DevBuf* b : bufs) b->release();
+  for (cudaEvent_t e : m->prof.pool) cudaEventDestroy(e);
   for (int i = 0; i < kStagingRing; ++i) {
     if (m->stg.host[i]) cudaFreeHost(m->stg.host[i]);
     if (m->stg.ev[i]) cudaEventDestroy(m->stg.ev[i]);
@@ -561,7 +612,7 @@ int cs_kv_alloc(const cs_model* m, int num_pages, int page_size, int max_seqs, i
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&kv->upload_ev, cudaEventDisableTiming);
   if (e != cudaSuccess) { rc = cuda_fail(e, "kv page table"); cs_kv_free(kv); return rc; }
   std::memset(kv->table_host, 0, tbytes);
-  if (!make_tensor_map_bf16(&kv->tm_pool, kv->pool, rows, m->d.head_dim, kPageSize, 64, true)) {
+  if (!make_tensor_map_16b(&kv->tm_pool, kv->pool, rows, m->d.head_dim, kPageSize, 64, true, true)) {
     g_cuda_error = "cuTensorMapEncodeTiled failed for the kv pool";
     cs_kv_free(kv);
     return CS_ECUDA;
@@ -620,7 +671,7 @@ int cs_kv_fill(cs_kv* kv, int seq, int layer, const uint16_t* host_k, const uint
   CS_CUDA(launch_kv_scatter(tk, tv, static_cast<int>(row), nullptr, nullptr, seq, 0, kv->table_dev,
                             kv->max_pages_per_seq, kv->pool + static_cast<size_t>(2 * layer) * kv->plane_elems,
                             kv->pool + static_cast<size_t>(2 * layer + 1) * kv->plane_elems, d.n_kv_heads, d.head_dim,
-                            kPageSize, c, s));
+                            kPageSize, c, 0, s));
   CS_CUDA(cudaStreamSynchronize(s));
   return CS_OK;
 }
@@ -672,14 +723,14 @@ int cs_verify_steps(cs_model* m, const cs_kv* ckv, const int32_t* seq_ids, int B
   float* x = static_cast<float*>(m->x.p);
   uint16_t* h_last = static_cast<uint16_t*>(m->h_last.p);
   const int B_all = ((B + 63) / 64) * 64;
-  CS_CUDA(launch_last_rows_norm(x, dev_meta + L.off_cu, m->final_norm, h_last, B, B_all, d.d_model, d.rms_eps, s));
+  CS_STEP(kProfNorm, launch_last_rows_norm(x, dev_meta + L.off_cu, m->final_norm, h_last, B, B_all, d.d_model, d.rms_eps, s));
   CUtensorMap tm_h;
   int tiles_per_cta;
   const int grid = lm_head_grid(d.vocab, &tiles_per_cta);
   for (int b0 = 0; b0 < B; b0 += 64) {
     const int bc = std::min(64, B - b0);
     const int bp = lm_head_batch_pad(bc);
-    if (!make_tensor_map_bf16(&tm_h, h_last, B_all, d.d_model, bp, 64, true)) {
+    if (!make_tensor_map_16b(&tm_h, h_last, B_all, d.d_model, bp, 64, true, false)) {
       g_cuda_error = "cuTensorMapEncodeTiled failed for the last-position hidden states";
       return CS_ECUDA;
     }
@@ -687,9 +738,9 @@ int cs_verify_steps(cs_model* m, const cs_kv* ckv, const int32_t* seq_ids, int B
     float* part_sum = part_max + kNumSMs * 64;
     float* vlog = static_cast<float*>(m->vlogits.p) + static_cast<size_t>(b0) * 8;
     float* logits = m->keep_logits ? static_cast<float*>(m->logits.p) + static_cast<size_t>(b0) * d.vocab : nullptr;
-    CS_CUDA(launch_lm_head(m->tm_lm, tm_h, b0, bc, bp, d.d_model, d.vocab, verdict_ids, n_verdict, part_max, part_sum,
+    CS_STEP(kProfLmHead, launch_lm_head(m->tm_lm, tm_h, b0, bc, bp, d.d_model, d.vocab, verdict_ids, n_verdict, part_max, part_sum,
                            vlog, logits, m->status, s));
-    CS_CUDA(launch_gate(part_max, part_sum, grid, bp, vlog, n_verdict, bc, tau, out_conf + b0, out_accept + b0,
+    CS_STEP(kProfGate, launch_gate(part_max, part_sum, grid, bp, vlog, n_verdict, bc, tau, out_conf + b0, out_accept + b0,
                         out_verdict ? out_verdict + b0 : nullptr, static_cast<float*>(m->lse.p) + b0, s));
   }
   m->last_B = B;
@@ -736,7 +787,29 @@ int cs_last_status(cs_model* m, void* stream) {
   return (v & 1u) ? CS_ETIMEOUT : CS_OK;
 }
 
-int cs_gemm_bf16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* out, int M, int N, int K,
+int cs_profile(cs_model* m, int enable) {
+  if (!m) return CS_EINVAL;
+  m->prof.on = enable != 0;
+  m->prof.used = 0;
+  return CS_OK;
+}
+
+int cs_profile_read(cs_model* m, float* ms_out, int32_t* launches_out, int n_classes) {
+  if (!m || !ms_out || !launches_out || n_classes < kProfClasses) return CS_EINVAL;
+  for (int c = 0; c < n_classes; ++c) { ms_out[c] = 0.f; launches_out[c] = 0; }
+  Prof& p = m->prof;
+  for (size_t i = 0; i < p.used; ++i) {
+    CS_CUDA(cudaEventSynchronize(p.pool[2 * i + 1]));
+    float ms = 0.f;
+    CS_CUDA(cudaEventElapsedTime(&ms, p.pool[2 * i], p.pool[2 * i + 1]));
+    ms_out[p.cls[i]] += ms;
+    launches_out[p.cls[i]] += 1;
+  }
+  p.used = 0;
+  return CS_OK;
+}
+
+int cs_gemm_f16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* out, int M, int N, int K,
                  int epilogue, void* stream) {
   if (!a || !w || !out || M < 0 || N < 8 || K < 8 || (N % 8) || (K % 8) || epilogue < 0 || epilogue > 2)
     return CS_EINVAL;
@@ -752,7 +825,7 @@ int cs_gemm_bf16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void*
     g_cuda_error = "cuTensorMapEncodeTiled failed";
     return CS_ECUDA;
   }
-  CS_CUDA(gemm_bf16(ta, tb, w2 ? &tb2 : nullptr, out, M, N, K, epilogue, g_test_status,
+  CS_CUDA(gemm_f16(ta, tb, w2 ? &tb2 : nullptr, out, M, N, K, epilogue, g_test_status,
                     static_cast<cudaStream_t>(stream)));
   return CS_OK;
 }

@@ -41,10 +41,10 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                : "r"(addr));
 }
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1) {
   asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
       "{%0, %1, %2, %3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
@@ -173,6 +173,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
     if (!mbar_wait(&full_bar[stage], phase, abort_flag, p.status)) { ok = false; break; }
     const uint32_t sk = smem_u32(smem + stage * L::kStageBytes);
     const uint32_t sv = sk + L::kTileBytes;
+    const bool cached = t < ctx_tiles;
 
     // S = Q K^T for 64 keys: 8 key groups of 8.
     float s[kKTile / 8][4];
@@ -184,8 +185,11 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       for (int j = 0; j < HD / 32; ++j) {
         uint32_t b0, b1, b2, b3;
         ldsm_x4(sk + tile_offset<HD>(key, j * 32 + (lane >> 3) * 8), b0, b1, b2, b3);
-        mma_bf16(s[nt], qf[2 * j][0], qf[2 * j][1], qf[2 * j][2], qf[2 * j][3], b0, b1);
-        mma_bf16(s[nt], qf[2 * j + 1][0], qf[2 * j + 1][1], qf[2 * j + 1][2], qf[2 * j + 1][3], b2, b3);
+        if (cached) {  // cache pages hold bf16; the query and the step's own keys are fp16
+          b0 = bf16x2_to_f16x2(b0); b1 = bf16x2_to_f16x2(b1); b2 = bf16x2_to_f16x2(b2); b3 = bf16x2_to_f16x2(b3);
+        }
+        mma_f16(s[nt], qf[2 * j][0], qf[2 * j][1], qf[2 * j][2], qf[2 * j][3], b0, b1);
+        mma_f16(s[nt], qf[2 * j + 1][0], qf[2 * j + 1][1], qf[2 * j + 1][2], qf[2 * j + 1][3], b2, b3);
       }
     }
 
@@ -233,8 +237,8 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       const float p2 = fast_exp2(fmaf(s[nt][2], sc, -ref_hi)), p3 = fast_exp2(fmaf(s[nt][3], sc, -ref_hi));
       l_lo += p0 + p1;
       l_hi += p2 + p3;
-      pf[nt >> 1][(nt & 1) * 2] = pack_bf16x2(p0, p1);
-      pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16x2(p2, p3);
+      pf[nt >> 1][(nt & 1) * 2] = pack_f16x2(p0, p1);
+      pf[nt >> 1][(nt & 1) * 2 + 1] = pack_f16x2(p2, p3);
     }
 
     // O += P V
@@ -245,8 +249,11 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       for (int np = 0; np < HD / 16; ++np) {
         uint32_t b0, b1, b2, b3;
         ldsm_x4_t(sv + tile_offset<HD>(key, np * 16 + (lane >> 4) * 8), b0, b1, b2, b3);
-        mma_bf16(o[2 * np], pf[ks][0], pf[ks][1], pf[ks][2], pf[ks][3], b0, b1);
-        mma_bf16(o[2 * np + 1], pf[ks][0], pf[ks][1], pf[ks][2], pf[ks][3], b2, b3);
+        if (cached) {
+          b0 = bf16x2_to_f16x2(b0); b1 = bf16x2_to_f16x2(b1); b2 = bf16x2_to_f16x2(b2); b3 = bf16x2_to_f16x2(b3);
+        }
+        mma_f16(o[2 * np], pf[ks][0], pf[ks][1], pf[ks][2], pf[ks][3], b0, b1);
+        mma_f16(o[2 * np + 1], pf[ks][0], pf[ks][1], pf[ks][2], pf[ks][3], b2, b3);
       }
     }
     __syncwarp();
@@ -267,13 +274,13 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       uint16_t* dst = p.out + static_cast<size_t>(tok0 + p_lo) * q_dim + (it.kv_head * G + (r_lo - p_lo * G)) * HD;
 #pragma unroll
       for (int i = 0; i < HD / 8; ++i)
-        *reinterpret_cast<uint32_t*>(dst + i * 8 + 2 * tq) = pack_bf16x2(o[i][0] * inv_lo, o[i][1] * inv_lo);
+        *reinterpret_cast<uint32_t*>(dst + i * 8 + 2 * tq) = pack_f16x2(o[i][0] * inv_lo, o[i][1] * inv_lo);
     }
     if (r_hi < rows_total) {
       uint16_t* dst = p.out + static_cast<size_t>(tok0 + p_hi) * q_dim + (it.kv_head * G + (r_hi - p_hi * G)) * HD;
 #pragma unroll
       for (int i = 0; i < HD / 8; ++i)
-        *reinterpret_cast<uint32_t*>(dst + i * 8 + 2 * tq) = pack_bf16x2(o[i][2] * inv_hi, o[i][3] * inv_hi);
+        *reinterpret_cast<uint32_t*>(dst + i * 8 + 2 * tq) = pack_f16x2(o[i][2] * inv_hi, o[i][3] * inv_hi);
     }
   } else {
     const int row_lo = warp * 16 + g, row_hi = row_lo + 8;
@@ -319,7 +326,7 @@ __global__ void attention_merge_kernel(const AttnParams p, const AttnMerge* __re
     const float inv = 1.f / l;
     const int pos = r / G;
     uint16_t* dst = p.out + static_cast<size_t>(tok0 + pos) * q_dim + (mg.kv_head * G + (r - pos * G)) * HD + c;
-    *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+    *reinterpret_cast<uint2*>(dst) = make_uint2(pack_f16x2(acc.x * inv, acc.y * inv), pack_f16x2(acc.z * inv, acc.w * inv));
   }
 }
 

@@ -43,7 +43,7 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
   for (int i = lane; i < d / 4; i += 32) {
     const float4 v = xr[i];
     const float4 g = g4[i];
-    o[i] = make_uint2(pack_bf16x2(v.x * r * g.x, v.y * r * g.y), pack_bf16x2(v.z * r * g.z, v.w * r * g.w));
+    o[i] = make_uint2(pack_f16x2(v.x * r * g.x, v.y * r * g.y), pack_f16x2(v.z * r * g.z, v.w * r * g.w));
   }
 }
 
@@ -72,9 +72,9 @@ __global__ void rope_apply_kernel(uint16_t* __restrict__ qkv, const float2* __re
   uint32_t* hi = reinterpret_cast<uint32_t*>(qkv + static_cast<size_t>(t) * n_qkv + head * hd + half + j);
   const uint32_t a = *lo, b = *hi;
   const float2 cs0 = table[t * half + j], cs1 = table[t * half + j + 1];
-  const float a0 = bf16_lo(a), a1 = bf16_hi(a), b0 = bf16_lo(b), b1 = bf16_hi(b);
-  *lo = pack_bf16x2(a0 * cs0.x - b0 * cs0.y, a1 * cs1.x - b1 * cs1.y);
-  *hi = pack_bf16x2(b0 * cs0.x + a0 * cs0.y, b1 * cs1.x + a1 * cs1.y);
+  const float2 av = unpack_f16x2(a), bv = unpack_f16x2(b);
+  *lo = pack_f16x2(av.x * cs0.x - bv.x * cs0.y, av.y * cs1.x - bv.y * cs1.y);
+  *hi = pack_f16x2(bv.x * cs0.x + av.x * cs0.y, bv.y * cs1.x + av.y * cs1.y);
 }
 
 // Thread per 16 bytes of a K row and of a V row.
@@ -83,7 +83,7 @@ __global__ void kv_scatter_kernel(const uint16_t* __restrict__ src_k, const uint
                                   const int32_t* __restrict__ tok_pos, int const_seq, int pos0,
                                   const int32_t* __restrict__ page_table,
                                   int max_pages_per_seq, uint16_t* __restrict__ pool_k, uint16_t* __restrict__ pool_v,
-                                  int n_kv_heads, int hd, int page_size, int T) {
+                                  int n_kv_heads, int hd, int page_size, int T, int src_is_f16) {
   const int chunks = n_kv_heads * hd / 8;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= T * chunks) return;
@@ -97,11 +97,31 @@ __global__ void kv_scatter_kernel(const uint16_t* __restrict__ src_k, const uint
   const int slot = pos % page_size;
   const size_t dst = ((static_cast<size_t>(page) * n_kv_heads + head) * page_size + slot) * hd + e;
   const size_t src = static_cast<size_t>(t) * row_stride + c * 8;
-  *reinterpret_cast<uint4*>(pool_k + dst) = *reinterpret_cast<const uint4*>(src_k + src);
-  *reinterpret_cast<uint4*>(pool_v + dst) = *reinterpret_cast<const uint4*>(src_v + src);
+  uint4 k = *reinterpret_cast<const uint4*>(src_k + src);
+  uint4 v = *reinterpret_cast<const uint4*>(src_v + src);
+  if (src_is_f16) {  // the cache format is bf16: round the fp16 activations
+    k = make_uint4(f16x2_to_bf16x2(k.x), f16x2_to_bf16x2(k.y), f16x2_to_bf16x2(k.z), f16x2_to_bf16x2(k.w));
+    v = make_uint4(f16x2_to_bf16x2(v.x), f16x2_to_bf16x2(v.y), f16x2_to_bf16x2(v.z), f16x2_to_bf16x2(v.w));
+  }
+  *reinterpret_cast<uint4*>(pool_k + dst) = k;
+  *reinterpret_cast<uint4*>(pool_v + dst) = v;
+}
+
+// In-place re-encoding of bf16 bit patterns as fp16 (same size). Exact for magnitudes in [2^-14, 65504];
+// smaller values round to the fp16 subnormal grid (absolute error <= 2^-25).
+__global__ void bf16_to_f16_kernel(uint32_t* __restrict__ p, size_t n_pairs) {
+  for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n_pairs;
+       i += static_cast<size_t>(gridDim.x) * blockDim.x)
+    p[i] = bf16x2_to_f16x2(p[i]);
 }
 
 }  // namespace
+
+cudaError_t launch_bf16_to_f16(uint16_t* p, size_t n, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  bf16_to_f16_kernel<<<1184, 256, 0, s>>>(reinterpret_cast<uint32_t*>(p), n / 2);
+  return cudaGetLastError();
+}
 
 void count_launch(int n) { g_launches += n; }
 int64_t take_launch_count() {
@@ -149,12 +169,12 @@ cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int 
                               const int32_t* tok_pos, int const_seq, int pos0, const int32_t* page_table,
                               int max_pages_per_seq,
                               uint16_t* pool_k_plane, uint16_t* pool_v_plane, int n_kv_heads, int hd, int page_size,
-                              int T, cudaStream_t s) {
+                              int T, int src_is_f16, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   const int n = T * n_kv_heads * hd / 8;
   kv_scatter_kernel<<<(n + 255) / 256, 256, 0, s>>>(src_k, src_v, row_stride, tok_seq, tok_pos, const_seq, pos0, page_table,
                                                     max_pages_per_seq, pool_k_plane, pool_v_plane, n_kv_heads, hd,
-                                                    page_size, T);
+                                                    page_size, T, src_is_f16);
   count_launch();
   return cudaGetLastError();
 }

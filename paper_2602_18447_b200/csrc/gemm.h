@@ -1,4 +1,4 @@
-// Host interface of the tcgen05 projection GEMM.
+// Host interface of the tcgen05 projection GEMM (fp16 operands, fp32 accumulation).
 #pragma once
 
 #include <cuda.h>
@@ -8,18 +8,19 @@
 namespace cs {
 
 enum GemmEpilogue {
-  kEpiStoreBf16 = 0,  // out bf16 [M,N] = a * w^T
+  kEpiStoreF16 = 0,  // out fp16 [M,N] = a * w^T
   kEpiResidAdd = 1,   // out fp32 [M,N] += a * w^T   (atomic adds, k-range split over the SMs)
-  kEpiSwiGLU = 2      // out bf16 [M,N] = silu(a * w^T) * (a * w2^T)
+  kEpiSwiGLU = 2      // out fp16 [M,N] = silu(a * w^T) * (a * w2^T)
 };
 
-// 2D bf16 tensor map over a row-major [rows, cols] matrix; box = [box_rows, box_cols].
-bool make_tensor_map_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
-                          uint32_t box_cols, bool swizzle128);
-// Tensor map of a GEMM operand ([rows, k] bf16, K-major): 128-row x 64-column boxes, 128-byte swizzle.
+// 2D tensor map over a row-major [rows, cols] matrix of 16-bit floats (fp16, or bf16 for the kv cache);
+// box = [box_rows, box_cols].
+bool make_tensor_map_16b(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                         uint32_t box_cols, bool swizzle128, bool is_bf16);
+// Tensor map of a GEMM operand ([rows, k] fp16, K-major): 128-row x 64-column boxes, 128-byte swizzle.
 bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k);
 
-cudaError_t gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,
+cudaError_t gemm_f16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,
                       int K, int epilogue, uint32_t* status, cudaStream_t stream);
 
 }  // namespace cs

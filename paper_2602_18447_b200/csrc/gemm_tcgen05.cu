@@ -1,4 +1,4 @@
-// Projection GEMMs of the decoder layers: out = a[M,K] * w[N,K]^T, bf16 in, fp32 accumulate in TMEM.
+// Projection GEMMs of the decoder layers: out = a[M,K] * w[N,K]^T, fp16 in, fp32 accumulate in TMEM.
 //
 // One persistent CTA per SM. Warp 0 feeds a ring of shared-memory stages with TMA (128-byte swizzle), warp 1
 // issues tcgen05.mma into one of two TMEM accumulators, warps 2-5 drain the other accumulator (tcgen05.ld)
@@ -6,7 +6,7 @@
 //
 // Work is measured in k-blocks (128 x BN x 64 products). Each CTA owns a contiguous range of k-blocks in the
 // order (n tile, m tile, k); a range may start or end inside a tile. For the two epilogues that need the whole
-// sum (bf16 store, SwiGLU) the ranges are whole tiles. For the residual epilogue (x += a * w^T, fp32) the
+// sum (fp16 store, SwiGLU) the ranges are whole tiles. For the residual epilogue (x += a * w^T, fp32) the
 // range is cut evenly over the SMs whatever the tile boundaries are, and every piece is added into x with
 // vector atomics, which is what lets the narrow O and down projections fill all SMs.
 #include "gemm.h"
@@ -55,13 +55,13 @@ __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                  const __grid_constant__ CUtensorMap tm_b2, void* __restrict__ out, int M, int N, int m_tiles,
                  int kblocks, int total_units, int units_per_cta, uint32_t* status) {
   using L = GemmSmem<BN>;
   constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
   constexpr uint32_t kTmemCols = 2 * BN;
-  constexpr uint32_t kIdesc = umma_idesc_bf16(BM, BN);
+  constexpr uint32_t kIdesc = umma_idesc_f16(BM, BN);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -157,7 +157,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           const uint64_t bdesc = umma_desc_k128(sa + kABytes);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
-            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (i | k) != 0);
+            umma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (i | k) != 0);
           umma_commit(&empty_bar[stage]);
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
@@ -186,7 +186,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       uint32_t r[32];
       if (EPI == kEpiSwiGLU) {
         uint32_t r2[32];
-        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + static_cast<size_t>(row) * N;
+        __half* o = reinterpret_cast<__half*>(out) + static_cast<size_t>(row) * N;
 #pragma unroll 1
         for (int c = 0; c < OUT_BN / 32; ++c) {
           tmem_ld_32x32(t_row + c * 32, r);
@@ -197,7 +197,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           for (int j = 0; j < 16; ++j) {
             const float g0 = __uint_as_float(r[2 * j]), g1 = __uint_as_float(r[2 * j + 1]);
             const float u0 = __uint_as_float(r2[2 * j]), u1 = __uint_as_float(r2[2 * j + 1]);
-            p[j] = pack_bf16x2(silu_f(g0) * u0, silu_f(g1) * u1);
+            p[j] = pack_f16x2(silu_f(g0) * u0, silu_f(g1) * u1);
           }
           const int col = n0 + c * 32;
           if (row_ok) {
@@ -206,8 +206,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
               if (col + j * 8 < N) st_v4(o + col + j * 8, p[4 * j], p[4 * j + 1], p[4 * j + 2], p[4 * j + 3]);
           }
         }
-      } else if (EPI == kEpiStoreBf16) {
-        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + static_cast<size_t>(row) * N;
+      } else if (EPI == kEpiStoreF16) {
+        __half* o = reinterpret_cast<__half*>(out) + static_cast<size_t>(row) * N;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           tmem_ld_32x32(t_row + c * 32, r);
@@ -217,10 +217,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 #pragma unroll
             for (int j = 0; j < 4; ++j)
               if (col + j * 8 < N)
-                st_v4(o + col + j * 8, pack_bf16x2(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1])),
-                      pack_bf16x2(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3])),
-                      pack_bf16x2(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5])),
-                      pack_bf16x2(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7])));
+                st_v4(o + col + j * 8, pack_f16x2(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1])),
+                      pack_f16x2(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3])),
+                      pack_f16x2(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5])),
+                      pack_f16x2(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7])));
           }
         }
       } else {
@@ -279,7 +279,7 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
   constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    cudaError_t e = cudaFuncSetAttribute(gemm_f16_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -298,7 +298,7 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
     grid = (tiles + tpc - 1) / tpc;
     upc = tpc * kblocks;
   }
-  gemm_bf16_kernel<BN, EPI><<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tb, tb2, out, M, N, m_tiles, kblocks, total,
+  gemm_f16_kernel<BN, EPI><<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tb, tb2, out, M, N, m_tiles, kblocks, total,
                                                                       upc, status);
   count_launch();
   return cudaGetLastError();
@@ -306,33 +306,33 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
 
 }  // namespace
 
-bool make_tensor_map_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
-                          uint32_t box_cols, bool swizzle128) {
+bool make_tensor_map_16b(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                         uint32_t box_cols, bool swizzle128, bool is_bf16) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {cols, rows};
   cuuint64_t strides[1] = {cols * 2};
   cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  CUresult r = fn(tm, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
 bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k) {
-  return make_tensor_map_bf16(tm, base, static_cast<uint64_t>(rows), static_cast<uint64_t>(k), 128, 64, true);
+  return make_tensor_map_16b(tm, base, static_cast<uint64_t>(rows), static_cast<uint64_t>(k), 128, 64, true, false);
 }
 
-cudaError_t gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,
+cudaError_t gemm_f16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,
                       int K, int epilogue, uint32_t* status, cudaStream_t stream) {
   if (M <= 0) return cudaSuccess;
   switch (epilogue) {
-    case kEpiStoreBf16:
+    case kEpiStoreF16:
       // Narrow outputs get 128-wide tiles so that the tile count comes closer to the SM count.
       if (((M + 127) / 128) * ((N + 255) / 256) < kNumSMs / 2 + 20)
-        return launch<128, kEpiStoreBf16>(ta, tb, tb, out, M, N, K, status, stream);
-      return launch<256, kEpiStoreBf16>(ta, tb, tb, out, M, N, K, status, stream);
+        return launch<128, kEpiStoreF16>(ta, tb, tb, out, M, N, K, status, stream);
+      return launch<256, kEpiStoreF16>(ta, tb, tb, out, M, N, K, status, stream);
     case kEpiResidAdd:
       return launch<256, kEpiResidAdd>(ta, tb, tb, out, M, N, K, status, stream);
     case kEpiSwiGLU:

@@ -29,8 +29,8 @@ struct AttnMerge {
 };
 
 struct AttnParams {
-  const uint16_t* qkv;      // [T, n_qkv] bf16: q heads, k heads, v heads (q, k already rotated)
-  uint16_t* out;            // [T, Hq*hd] bf16
+  const uint16_t* qkv;      // [T, n_qkv] fp16: q heads, k heads, v heads (q, k already rotated)
+  uint16_t* out;            // [T, Hq*hd] fp16
   const int32_t* cu_new;    // [B+1]
   const int32_t* ctx_len;   // [B]
   const int32_t* seq_id;    // [B]
@@ -61,7 +61,9 @@ cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int 
                               const int32_t* tok_pos, int const_seq, int pos0, const int32_t* page_table,
                               int max_pages_per_seq,
                               uint16_t* pool_k_plane, uint16_t* pool_v_plane, int n_kv_heads, int hd, int page_size,
-                              int T, cudaStream_t s);
+                              int T, int src_is_f16, cudaStream_t s);
+// Re-encode n bf16 values (n even) as fp16 in place.
+cudaError_t launch_bf16_to_f16(uint16_t* p, size_t n, cudaStream_t s);
 
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_pool, const CUtensorMap& tm_qkv,
                              const AttnItem* items, int n_items, const AttnMerge* merges, int n_merges,

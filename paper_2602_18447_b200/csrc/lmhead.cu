@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(kLmThreads, 1)
 lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const LmArgs a) {
   using L = LmSmem<NB>;
   constexpr uint32_t kTmemCols = (2 * NB < 32) ? 32 : 2 * NB;
-  constexpr uint32_t kIdesc = umma_idesc_bf16(kLmBM, NB);
+  constexpr uint32_t kIdesc = umma_idesc_f16(kLmBM, NB);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -130,7 +130,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
           const uint64_t bdesc = umma_desc_k128(sw + kLmWBytes);
 #pragma unroll
           for (int k = 0; k < kLmBK / 16; ++k)
-            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0);
+            umma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0);
           umma_commit(&empty_bar[stage]);
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
@@ -243,7 +243,7 @@ __global__ void last_rows_norm_kernel(const float* __restrict__ x, const int32_t
   for (int i = lane; i < d / 4; i += 32) {
     const float4 v = xr[i];
     const float4 g = g4[i];
-    o[i] = make_uint2(pack_bf16x2(v.x * r * g.x, v.y * r * g.y), pack_bf16x2(v.z * r * g.z, v.w * r * g.w));
+    o[i] = make_uint2(pack_f16x2(v.x * r * g.x, v.y * r * g.y), pack_f16x2(v.z * r * g.z, v.w * r * g.w));
   }
 }
 

@@ -5,18 +5,17 @@ import numpy as np
 import pytest
 
 from oracle import confspec_oracle as O
-from workloads import bf16_bits_from_f32
 
 pytestmark = pytest.mark.gpu
 
 
-def _bf16_randn(g, shape, std):
-    return bf16_bits_from_f32((std * g.standard_normal(shape)).astype(np.float32))
+def _f16_randn(g, shape, std):
+    return (std * g.standard_normal(shape)).astype(np.float16)
 
 
-def _to_dev(bits):
+def _to_dev(a):
     import torch
-    return torch.from_numpy(bits.view(np.int16)).cuda()
+    return torch.from_numpy(a).cuda()
 
 
 GEMM_SHAPES = [
@@ -36,24 +35,24 @@ def test_gemm_matches_oracle_matmul(M, N, K, epilogue):
     import torch
     from paper_2602_18447_b200 import binding as B
     g = np.random.default_rng(1000 + M + N + K + epilogue)
-    a = _bf16_randn(g, (M, K), 1.0)
-    w = _bf16_randn(g, (N, K), 0.05)
-    w2 = _bf16_randn(g, (N, K), 0.05)
-    af, wf, w2f = O.widen_bf16(a), O.widen_bf16(w), O.widen_bf16(w2)
+    a = _f16_randn(g, (M, K), 1.0)
+    w = _f16_randn(g, (N, K), 0.05)
+    w2 = _f16_randn(g, (N, K), 0.05)
+    af, wf, w2f = a.astype(np.float64), w.astype(np.float64), w2.astype(np.float64)
     da, dw, dw2 = _to_dev(a), _to_dev(w), _to_dev(w2)
     if epilogue == 1:
         x0 = g.standard_normal((M, N)).astype(np.float32)
         out = torch.from_numpy(x0.copy()).cuda()
         want = x0.astype(np.float64) + af @ wf.T
     else:
-        out = torch.full((M, N), -777.0, dtype=torch.bfloat16, device="cuda")
+        out = torch.full((M, N), -777.0, dtype=torch.float16, device="cuda")
         want = af @ wf.T if epilogue == 0 else O.silu(af @ wf.T) * (af @ w2f.T)
-    B.cs_gemm_bf16(da, dw, dw2 if epilogue == 2 else None, out, M, N, K, epilogue)
+    B.cs_gemm_f16(da, dw, dw2 if epilogue == 2 else None, out, M, N, K, epilogue)
     torch.cuda.synchronize()
     got = out.float().cpu().numpy().astype(np.float64)
     scale = float(np.abs(want).max())
-    # fp32 accumulation of exact bf16 products, then one rounding to the output type
-    tol = (2.0 ** -8) * np.abs(want) + 2e-5 * scale * (1 + K / 1024) if epilogue != 1 else 3e-5 * scale * (1 + K / 1024)
+    # fp32 accumulation of exact fp16 products, then one rounding to the output type
+    tol = (2.0 ** -11) * np.abs(want) + 2e-5 * scale * (1 + K / 1024) if epilogue != 1 else 3e-5 * scale * (1 + K / 1024)
     bad = np.abs(got - want) > tol
     assert not bad.any(), (int(bad.sum()), float(np.abs(got - want).max()), scale)
 
@@ -65,12 +64,12 @@ def test_rmsnorm_matches_oracle(rows, d):
     g = np.random.default_rng(rows * 7 + d)
     x = (g.standard_normal((rows, d)) * g.uniform(0.01, 30.0, size=(rows, 1))).astype(np.float32)
     gain = (1.0 + 0.2 * g.standard_normal(d)).astype(np.float32)
-    out = torch.empty((rows, d), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty((rows, d), dtype=torch.float16, device="cuda")
     B.cs_rmsnorm(torch.from_numpy(x).cuda(), torch.from_numpy(gain).cuda(), out, rows, d, 1e-6)
     torch.cuda.synchronize()
     want = O.rmsnorm(x.astype(np.float64), gain.astype(np.float64), 1e-6)
     got = out.float().cpu().numpy().astype(np.float64)
-    assert np.all(np.abs(got - want) <= (2.0 ** -8) * np.abs(want) + 1e-6)
+    assert np.all(np.abs(got - want) <= (2.0 ** -11) * np.abs(want) + 1e-6)
 
 
 def test_escalate_mask_matches_oracle_bit_exact():
