@@ -23,7 +23,7 @@ sys.path.insert(0, ROOT)
 
 import numpy as np  # noqa: E402
 
-from workloads import context_kv, get_config, make_batch, model_weights, page_assignment  # noqa: E402
+from workloads import context_kv, get_config, make_batch, model_weights, page_assignment, scaled_config  # noqa: E402
 
 METRIC = "verified_steps_per_s"
 UNIT = "steps/s"
@@ -306,7 +306,7 @@ def run_ours(args, cfg):
         "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16", "data": "synthetic",
         "tokens_per_s": all_tokens * K / (ms * 1e-3),
-        "config": {"workload": cfg.name, "model": cfg.model.name, "batch": cfg.batch, "new_tokens": counts["T"],
+        "config": {"workload": cfg.name, "model": cfg.model.name, "layers": cfg.model.n_layers, "batch": cfg.batch, "new_tokens": counts["T"],
                    "ctx_tokens": int(batch.ctx_lens.sum()), "tau": cfg.tau, "page_size": cfg.page_size,
                    "l2": "inputs larger than L2 (3.1 GB of weights streamed every step)",
                    "replicas": world},
@@ -343,8 +343,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="run a reduced-depth copy of the workload (for profiler captures of single kernels); "
+                         "not a benchmark configuration")
     args = ap.parse_args()
     cfg = get_config(args.workload)
+    if args.layers is not None:
+        cfg = scaled_config(args.workload, n_layers=args.layers)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
