@@ -156,31 +156,30 @@ struct BatchLayout {
   int n_items = 0, n_merges = 0, n_slots = 0;
 };
 
-// Splits the attention of every (step, kv head, 64-row query tile) into key-tile ranges of similar length so
-// that the grid is a few times the SM count, longest ranges first.
+// Splits the attention of every (step, kv head, query tile of 128 / G tokens) into key-tile ranges of similar
+// length so that the grid is about twice the SM count, longest ranges first.
 void build_attention_work(const cs_model* m, int B, const int32_t* lens, const int32_t* ctx, std::vector<AttnItem>& items,
                           std::vector<AttnMerge>& merges, int* n_slots) {
   const int G = m->d.n_q_heads / m->d.n_kv_heads;
+  const int ntok = 128 / G;
   long total_tiles = 0;
   for (int i = 0; i < B; ++i) {
-    const int rows = lens[i] * G;
     const int ctx_tiles = (ctx[i] + 63) / 64;
-    for (int q0 = 0; q0 < rows; q0 += 64) {
-      const int p_max = std::min(lens[i] - 1, (q0 + 63) / G);
+    for (int q0 = 0; q0 < lens[i]; q0 += ntok) {
+      const int p_max = std::min(lens[i] - 1, q0 + ntok - 1);
       total_tiles += static_cast<long>(ctx_tiles + p_max / 64 + 1) * m->d.n_kv_heads;
     }
   }
-  const long target_items = 3L * kNumSMs;
-  const int chunk = static_cast<int>(std::max<long>(8, (total_tiles + target_items - 1) / target_items));
+  const long target_items = 2L * kNumSMs;
+  const int chunk = static_cast<int>(std::max<long>(6, (total_tiles + target_items - 1) / target_items));
   items.clear();
   merges.clear();
   int slots = 0;
   for (int i = 0; i < B; ++i) {
-    const int rows = lens[i] * G;
     const int ctx_tiles = (ctx[i] + 63) / 64;
     for (int h = 0; h < m->d.n_kv_heads; ++h) {
-      for (int q0 = 0; q0 < rows; q0 += 64) {
-        const int p_max = std::min(lens[i] - 1, (q0 + 63) / G);
+      for (int q0 = 0; q0 < lens[i]; q0 += ntok) {
+        const int p_max = std::min(lens[i] - 1, q0 + ntok - 1);
         const int nt = ctx_tiles + p_max / 64 + 1;
         int splits = (nt + chunk - 1) / chunk;
         if (nt < chunk + chunk / 2) splits = 1;
@@ -273,10 +272,13 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   uint16_t* hmlp = static_cast<uint16_t*>(m->hmlp.p);
   float2* rope = static_cast<float2*>(m->rope.p);
 
-  CUtensorMap tm_a, tm_o, tm_h, tm_qkv_attn;
+  CUtensorMap tm_a, tm_o, tm_h, tm_qkv_attn, tm_q3d;
+  const int group = d.n_q_heads / d.n_kv_heads;
   if (!make_gemm_operand_map(&tm_a, a, T, d.d_model) || !make_gemm_operand_map(&tm_o, attn_o, T, m->q_dim) ||
       !make_gemm_operand_map(&tm_h, hmlp, T, d.d_ffn) ||
-      !make_tensor_map_16b(&tm_qkv_attn, qkv, T, m->n_qkv, kPageSize, 64, true, false)) {
+      !make_tensor_map_16b(&tm_qkv_attn, qkv, T, m->n_qkv, kPageSize, 64, true, false) ||
+      !make_tensor_map_heads3d(&tm_q3d, qkv, T, d.n_q_heads + 2 * d.n_kv_heads, d.head_dim, m->n_qkv, 128 / group,
+                               group)) {
     g_cuda_error = "cuTensorMapEncodeTiled failed for an activation buffer";
     return CS_ECUDA;
   }
@@ -309,7 +311,7 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
     CS_STEP(kProfRope, launch_rope_apply(qkv, rope, T, m->n_qkv, d.n_q_heads + d.n_kv_heads, d.head_dim, s));
     ap.k_row_base = (2 * l) * plane_rows;
     ap.v_row_base = (2 * l + 1) * plane_rows;
-    CS_STEP(kProfAttn, launch_attention(ap, kv->tm_pool, tm_qkv_attn, d_items, L.n_items, d_merges, L.n_merges, s));
+    CS_STEP(kProfAttn, launch_attention(ap, kv->tm_pool, tm_qkv_attn, tm_q3d, d_items, L.n_items, d_merges, L.n_merges, s));
     if (append_kv) {
       CS_STEP(kProfOther, launch_kv_scatter(qkv + m->q_dim, qkv + m->q_dim + m->kv_dim, m->n_qkv, d_tseq, d_pos, 0, 0,
                                 append_kv->table_dev, append_kv->max_pages_per_seq,
@@ -388,8 +390,8 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   int rc;
   if ((rc = ensure_workspace(m, B, L.T))) return rc;
   const int hd = m->d.head_dim;
-  if ((rc = m->attn_part_o.ensure(static_cast<size_t>(std::max(1, n_slots)) * 64 * hd * 4))) return rc;
-  if ((rc = m->attn_part_ml.ensure(static_cast<size_t>(std::max(1, n_slots)) * 64 * 2 * 4))) return rc;
+  if ((rc = m->attn_part_o.ensure(static_cast<size_t>(std::max(1, n_slots)) * 128 * hd * 4))) return rc;
+  if ((rc = m->attn_part_ml.ensure(static_cast<size_t>(std::max(1, n_slots)) * 128 * 2 * 4))) return rc;
   if ((rc = m->stg.dev.ensure(L.total * 4))) return rc;
   int slot;
   if ((rc = staging_slot(m->stg, L.total, &slot))) return rc;

@@ -17,6 +17,11 @@ enum GemmEpilogue {
 // box = [box_rows, box_cols].
 bool make_tensor_map_16b(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
                          uint32_t box_cols, bool swizzle128, bool is_bf16);
+// 3D fp16 tensor map over a row-major [tokens, heads, head_dim] view (token stride = row_elems elements):
+// box = [box_tokens, box_heads, 64], 128-byte swizzle. Used to fetch a query tile whose rows are
+// (token, head-in-group) pairs.
+bool make_tensor_map_heads3d(CUtensorMap* tm, const void* base, uint64_t tokens, uint64_t heads, uint32_t head_dim,
+                             uint64_t row_elems, uint32_t box_tokens, uint32_t box_heads);
 // Tensor map of a GEMM operand ([rows, k] fp16, K-major): 128-row x 64-column boxes, 128-byte swizzle.
 bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k);
 

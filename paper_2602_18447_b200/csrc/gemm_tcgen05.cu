@@ -320,6 +320,20 @@ bool make_tensor_map_16b(CUtensorMap* tm, const void* base, uint64_t rows, uint6
   return r == CUDA_SUCCESS;
 }
 
+bool make_tensor_map_heads3d(CUtensorMap* tm, const void* base, uint64_t tokens, uint64_t heads, uint32_t head_dim,
+                             uint64_t row_elems, uint32_t box_tokens, uint32_t box_heads) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {head_dim, heads, tokens};
+  cuuint64_t strides[2] = {static_cast<cuuint64_t>(head_dim) * 2, row_elems * 2};
+  cuuint32_t box[3] = {64, box_heads, box_tokens};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k) {
   return make_tensor_map_16b(tm, base, static_cast<uint64_t>(rows), static_cast<uint64_t>(k), 128, 64, true, false);
 }

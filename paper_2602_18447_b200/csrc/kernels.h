@@ -9,14 +9,14 @@ namespace cs {
 
 constexpr int kNumSMs = 148;
 
-// One unit of attention work: a tile of 64 query rows of one (step, kv head) over a range of 64-key tiles.
-// Query rows of a (step, kv head) are the pairs (new position p, head-in-group g) flattened as p * G + g.
+// One unit of attention work: the query rows of 128 / G consecutive new tokens of one step for the G query
+// heads of one kv head (row = token * G + head-in-group, at most 128 rows), over a range of 64-key tiles.
 // Key tiles 0 .. ctx_tiles-1 cover the cached context (4 pages each), the following ones the step's own
 // new keys.
 struct AttnItem {
   int32_t step;       // index into the batch
   int32_t kv_head;
-  int32_t q_row0;     // first flattened query row of the tile (multiple of 64)
+  int32_t q_tok0;     // first new token of the query tile, relative to the step (multiple of 128 / G)
   int32_t tile_begin; // key tile range [tile_begin, tile_end)
   int32_t tile_end;
   int32_t slot;       // partial-result slot, or -1 when the range is the whole key sequence
@@ -25,7 +25,7 @@ struct AttnItem {
 
 // A group of partial results to merge: slots [slot0, slot0 + n_splits) belong to one query tile.
 struct AttnMerge {
-  int32_t step, kv_head, q_row0, slot0, n_splits, pad0, pad1, pad2;
+  int32_t step, kv_head, q_tok0, slot0, n_splits, pad0, pad1, pad2;
 };
 
 struct AttnParams {
@@ -39,8 +39,8 @@ struct AttnParams {
   int32_t n_q_heads, n_kv_heads, head_dim, n_qkv;
   int32_t k_row_base, v_row_base;  // first pool row of this layer's K and V planes
   float scale_log2e;        // log2(e) / sqrt(head_dim)
-  float* part_o;            // [slots, 64, hd] unnormalised partial outputs
-  float* part_ml;           // [slots, 64, 2]  running max (raw score units) and sum
+  float* part_o;            // [slots, 128, hd] unnormalised partial outputs
+  float* part_ml;           // [slots, 128, 2]  exponent reference (raw score units) and sum
   uint32_t* status;
 };
 
@@ -65,9 +65,11 @@ cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int 
 // Re-encode n bf16 values (n even) as fp16 in place.
 cudaError_t launch_bf16_to_f16(uint16_t* p, size_t n, cudaStream_t s);
 
+// tm_pool: 2D map of the bf16 cache (16-row x 64-column boxes); tm_qkv: 2D map of the fp16 qkv workspace with
+// the same box; tm_q3d: 3D map (head_dim, head, token) of the same workspace with box (64, G, 128 / G).
 cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_pool, const CUtensorMap& tm_qkv,
-                             const AttnItem* items, int n_items, const AttnMerge* merges, int n_merges,
-                             cudaStream_t s);
+                             const CUtensorMap& tm_q3d, const AttnItem* items, int n_items, const AttnMerge* merges,
+                             int n_merges, cudaStream_t s);
 
 // h[b] = RMSNorm(x[last_row[b]]) as bf16 [B_pad, d]; rows B..B_pad-1 are zeroed.
 cudaError_t launch_last_rows_norm(const float* x, const int32_t* cu_new, const float* gain, uint16_t* h, int B,
