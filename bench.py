@@ -176,6 +176,28 @@ def run_reference(args, cfg):
 
 
 # ------------------------------------------------------------------------------------------------
+# rank aggregation (replicas only: no collective on the data path, only on the timings)
+# ------------------------------------------------------------------------------------------------
+def aggregate_over_ranks(ms: float, ms_e2e: float, n_steps: int, n_tokens: int, device=None):
+    """Whole-job figures of N independent replicas: the slowest rank's device times (MAX) and the units all
+    ranks processed (SUM). Without an initialised process group it returns the inputs unchanged."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms), float(ms_e2e), float(n_steps), float(n_tokens)
+    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    nb = torch.tensor([n_steps, n_tokens], dtype=torch.float64, device=device)
+    dist.all_reduce(nb, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), float(nb[0]), float(nb[1])
+
+
+def replica_seed(cfg, rank: int) -> int:
+    """Every replica verifies its own seeded batch."""
+    return cfg.seed + 7919 * rank
+
+
+# ------------------------------------------------------------------------------------------------
 # CUDA path
 # ------------------------------------------------------------------------------------------------
 def run_ours(args, cfg):
@@ -197,7 +219,7 @@ def run_ours(args, cfg):
             dist.barrier()
 
     weights = model_weights(cfg.model, cfg.seed)
-    batch = make_batch(cfg, seed=cfg.seed + 7919 * rank)       # each replica verifies its own batch
+    batch = make_batch(cfg, seed=replica_seed(cfg, rank))
     ses = VerifySession(cfg, weights, batch, device=f"cuda:{local}")
     total, pages = page_assignment(cfg, batch.ctx_lens)
     if cfg.ctx_kv == "prefill":
@@ -263,15 +285,8 @@ def run_ours(args, cfg):
     sampler.stop()
     clocks = sampler.summary(t_wall0, t_wall1)
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
-        nb = torch.tensor([batch.n_steps, batch.n_tokens], dtype=torch.float64, device="cuda")
-        dist.all_reduce(nb, op=dist.ReduceOp.SUM)
-        all_steps, all_tokens = float(nb[0]), float(nb[1])
-    else:
-        all_steps, all_tokens = float(batch.n_steps), float(batch.n_tokens)
+    ms, ms_e2e, all_steps, all_tokens = aggregate_over_ranks(
+        ms, ms_e2e, batch.n_steps, batch.n_tokens, device="cuda" if world > 1 else None)
 
     peaks, peak_kind = load_peaks()
     tensor_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))   # fp16 and bf16 share the peak
