@@ -41,7 +41,7 @@ struct LayerDev {
 struct DevBuf {
   void* p = nullptr;
   size_t cap = 0;
-  int ensure(size_t bytes) {
+  int ensure(size_t bytes, bool zero = false) {
     if (bytes <= cap) return CS_OK;
     if (p) {
       cudaDeviceSynchronize();
@@ -52,6 +52,7 @@ struct DevBuf {
     const size_t want = bytes + bytes / 4 + 256;
     cudaError_t e = cudaMalloc(&p, want);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(workspace)");
+    if (zero && (e = cudaMemset(p, 0, want)) != cudaSuccess) return cuda_fail(e, "cudaMemset(workspace)");
     cap = want;
     return CS_OK;
   }
@@ -93,7 +94,7 @@ struct cs_model {
   std::vector<void*> owned;
   CUtensorMap tm_lm;
   // workspace
-  DevBuf x, a, qkv, attn_o, hmlp, rope, h_last, lm_part, vlogits, logits, lse, attn_part_o, attn_part_ml;
+  DevBuf x, a, qkv, attn_o, hmlp, rope, h_last, lm_part, vlogits, logits, lse, attn_part_o, attn_part_ml, attn_counters;
   uint32_t* status = nullptr;
   Staging stg;
   bool keep_logits = false;
@@ -152,50 +153,87 @@ int staging_slot(Staging& st, size_t ints, int* slot_out) {
 
 struct BatchLayout {
   int B = 0, T = 0;
-  size_t off_cu, off_ctx, off_seq, off_pos, off_tseq, off_tok, off_items, off_merges, total;
-  int n_items = 0, n_merges = 0, n_slots = 0;
+  size_t off_cu, off_ctx, off_seq, off_pos, off_tseq, off_tok, off_items, total;
+  int n_items = 0, n_slots = 0;
 };
 
-// Splits the attention of every (step, kv head, query tile of 128 / G tokens) into key-tile ranges of similar
-// length so that the grid is about twice the SM count, longest ranges first.
+// Cost of an attention work item in key tiles: the tiles themselves plus the fixed part of a CTA (set-up, Q load,
+// pipeline fill, epilogue), and what the last piece of a split query tile adds by combining the partial results.
+constexpr double kAttnItemFixed = 3.0;
+constexpr double kAttnMergeFixed = 1.0;
+constexpr double kAttnMergePerSplit = 0.4;
+
+// Time at which the last SM finishes when the items, sorted by decreasing cost, are handed to whichever of
+// `machines` SMs is free first (what the hardware does with one CTA per SM and the grid in that order).
+double list_schedule_makespan(std::vector<double>& cost, int machines) {
+  std::sort(cost.begin(), cost.end(), std::greater<double>());
+  if (static_cast<int>(cost.size()) <= machines) return cost.empty() ? 0.0 : cost[0];
+  std::vector<double> heap(cost.begin(), cost.begin() + machines);   // min-heap of finish times
+  std::make_heap(heap.begin(), heap.end(), std::greater<double>());
+  for (size_t i = machines; i < cost.size(); ++i) {
+    std::pop_heap(heap.begin(), heap.end(), std::greater<double>());
+    heap.back() += cost[i];
+    std::push_heap(heap.begin(), heap.end(), std::greater<double>());
+  }
+  return *std::max_element(heap.begin(), heap.end());
+}
+
+// Work items of one attention launch: every (step, kv head, query tile of 128 / G tokens) over its key tiles,
+// long key ranges cut into pieces of at most `max_tiles` tiles. `max_tiles` is the candidate with the smallest
+// estimated finish time on the SMs; cutting is only worth it when it shortens the longest item by more than the
+// extra fixed cost and the combining step add.
 void build_attention_work(const cs_model* m, int B, const int32_t* lens, const int32_t* ctx, std::vector<AttnItem>& items,
-                          std::vector<AttnMerge>& merges, int* n_slots) {
+                          int* n_slots) {
   const int G = m->d.n_q_heads / m->d.n_kv_heads;
   const int ntok = 128 / G;
-  long total_tiles = 0;
+  const int max_splits = attention_max_splits();
+  struct Unit { int step, q0, nt; };
+  std::vector<Unit> units;
+  int longest = 1;
   for (int i = 0; i < B; ++i) {
-    const int ctx_tiles = (ctx[i] + 63) / 64;
+    const int ctx_tiles = (ctx[i] + 127) / 128;
     for (int q0 = 0; q0 < lens[i]; q0 += ntok) {
       const int p_max = std::min(lens[i] - 1, q0 + ntok - 1);
-      total_tiles += static_cast<long>(ctx_tiles + p_max / 64 + 1) * m->d.n_kv_heads;
+      const int nt = ctx_tiles + p_max / 128 + 1;
+      units.push_back(Unit{i, q0, nt});
+      longest = std::max(longest, nt);
     }
   }
-  const long target_items = 2L * kNumSMs;
-  const int chunk = static_cast<int>(std::max<long>(6, (total_tiles + target_items - 1) / target_items));
-  items.clear();
-  merges.clear();
-  int slots = 0;
-  for (int i = 0; i < B; ++i) {
-    const int ctx_tiles = (ctx[i] + 63) / 64;
-    for (int h = 0; h < m->d.n_kv_heads; ++h) {
-      for (int q0 = 0; q0 < lens[i]; q0 += ntok) {
-        const int p_max = std::min(lens[i] - 1, q0 + ntok - 1);
-        const int nt = ctx_tiles + p_max / 64 + 1;
-        int splits = (nt + chunk - 1) / chunk;
-        if (nt < chunk + chunk / 2) splits = 1;
-        if (splits <= 1) {
-          items.push_back(AttnItem{i, h, q0, 0, nt, -1, 0, 0});
-        } else {
-          merges.push_back(AttnMerge{i, h, q0, slots, splits, 0, 0, 0});
-          for (int s = 0; s < splits; ++s) {
-            const int b = static_cast<int>(static_cast<long>(nt) * s / splits);
-            const int e = static_cast<int>(static_cast<long>(nt) * (s + 1) / splits);
-            items.push_back(AttnItem{i, h, q0, b, e, slots++, 0, 0});
-          }
-        }
+  const int heads = m->d.n_kv_heads;
+  auto pieces = [&](int nt, int cap) { return std::min(max_splits, (nt + cap - 1) / cap); };
+  auto estimate = [&](int cap) {
+    std::vector<double> cost;
+    cost.reserve(units.size() * heads * 2);
+    for (const Unit& u : units) {
+      const int n = pieces(u.nt, cap);
+      for (int s = 0; s < n; ++s) {
+        const int len = static_cast<int>(static_cast<long>(u.nt) * (s + 1) / n - static_cast<long>(u.nt) * s / n);
+        double c = kAttnItemFixed + len;
+        if (n > 1 && s == n - 1) c += kAttnMergeFixed + kAttnMergePerSplit * n;
+        for (int h = 0; h < heads; ++h) cost.push_back(c);
       }
     }
+    return list_schedule_makespan(cost, kNumSMs);
+  };
+  int best_cap = longest;
+  double best = estimate(longest);
+  for (int k = 2; k <= 16 && longest / k >= 2; ++k) {
+    const int cap = (longest + k - 1) / k;
+    const double e = estimate(cap);
+    if (e < 0.97 * best) { best = e; best_cap = cap; }
   }
+  items.clear();
+  int slots = 0;
+  for (const Unit& u : units)
+    for (int h = 0; h < heads; ++h) {
+      const int n = pieces(u.nt, best_cap);
+      for (int s = 0; s < n; ++s) {
+        const int b = static_cast<int>(static_cast<long>(u.nt) * s / n);
+        const int e = static_cast<int>(static_cast<long>(u.nt) * (s + 1) / n);
+        items.push_back(AttnItem{u.step, h, u.q0, b, e, n > 1 ? slots + s : 0, n > 1 ? slots : 0, n});
+      }
+      if (n > 1) slots += n;
+    }
   std::stable_sort(items.begin(), items.end(), [](const AttnItem& a, const AttnItem& b) {
     return (a.tile_end - a.tile_begin) > (b.tile_end - b.tile_begin);
   });
@@ -263,7 +301,6 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   const int32_t* d_pos = dev_meta + L.off_pos;
   const int32_t* d_tseq = dev_meta + L.off_tseq;
   const AttnItem* d_items = reinterpret_cast<const AttnItem*>(dev_meta + L.off_items);
-  const AttnMerge* d_merges = reinterpret_cast<const AttnMerge*>(dev_meta + L.off_merges);
 
   float* x = static_cast<float*>(m->x.p);
   uint16_t* a = static_cast<uint16_t*>(m->a.p);
@@ -276,7 +313,7 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   const int group = d.n_q_heads / d.n_kv_heads;
   if (!make_gemm_operand_map(&tm_a, a, T, d.d_model) || !make_gemm_operand_map(&tm_o, attn_o, T, m->q_dim) ||
       !make_gemm_operand_map(&tm_h, hmlp, T, d.d_ffn) ||
-      !make_tensor_map_16b(&tm_qkv_attn, qkv, T, m->n_qkv, kPageSize, 64, true, false) ||
+      !make_kv_rows_map(&tm_qkv_attn, qkv, T, m->n_qkv, d.head_dim) ||
       !make_tensor_map_heads3d(&tm_q3d, qkv, T, d.n_q_heads + 2 * d.n_kv_heads, d.head_dim, m->n_qkv, 128 / group,
                                group)) {
     g_cuda_error = "cuTensorMapEncodeTiled failed for an activation buffer";
@@ -301,17 +338,18 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   ap.scale_log2e = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(d.head_dim)));
   ap.part_o = static_cast<float*>(m->attn_part_o.p);
   ap.part_ml = static_cast<float*>(m->attn_part_ml.p);
+  ap.counters = static_cast<int32_t*>(m->attn_counters.p);
   ap.status = m->status;
-  const int plane_rows = kv->num_pages * d.n_kv_heads * kPageSize;
+  const int plane_groups = kv->num_pages * d.n_kv_heads * kPageSize / 8;
 
   for (int l = 0; l < d.n_layers; ++l) {
     const LayerDev& lw = m->layers[l];
     CS_STEP(kProfNorm, launch_rmsnorm(x, lw.norm1, a, T, d.d_model, d.rms_eps, s));
     CS_STEP(kProfQkv, gemm_f16(tm_a, lw.tm_wqkv, nullptr, qkv, T, m->n_qkv, d.d_model, kEpiStoreF16, m->status, s));
     CS_STEP(kProfRope, launch_rope_apply(qkv, rope, T, m->n_qkv, d.n_q_heads + d.n_kv_heads, d.head_dim, s));
-    ap.k_row_base = (2 * l) * plane_rows;
-    ap.v_row_base = (2 * l + 1) * plane_rows;
-    CS_STEP(kProfAttn, launch_attention(ap, kv->tm_pool, tm_qkv_attn, tm_q3d, d_items, L.n_items, d_merges, L.n_merges, s));
+    ap.k_group_base = (2 * l) * plane_groups;
+    ap.v_group_base = (2 * l + 1) * plane_groups;
+    CS_STEP(kProfAttn, launch_attention(ap, kv->tm_pool, tm_qkv_attn, tm_q3d, d_items, L.n_items, s));
     if (append_kv) {
       CS_STEP(kProfOther, launch_kv_scatter(qkv + m->q_dim, qkv + m->q_dim + m->kv_dim, m->n_qkv, d_tseq, d_pos, 0, 0,
                                 append_kv->table_dev, append_kv->max_pages_per_seq,
@@ -333,7 +371,9 @@ int ensure_workspace(cs_model* m, int B, int T) {
   const size_t t = static_cast<size_t>(T);
   if ((rc = m->x.ensure(t * d.d_model * 4))) return rc;
   if ((rc = m->a.ensure(t * d.d_model * 2))) return rc;
-  if ((rc = m->qkv.ensure(t * m->n_qkv * 2))) return rc;
+  // A 128-row K/V box of the attention kernel may start at any of the T rows: the rows it reaches past the end
+  // must exist and be finite (they are masked, but they are multiplied), so the buffer is zeroed when it is made.
+  if ((rc = m->qkv.ensure((t + 128) * m->n_qkv * 2, true))) return rc;
   if ((rc = m->attn_o.ensure(t * m->q_dim * 2))) return rc;
   if ((rc = m->hmlp.ensure(t * d.d_ffn * 2))) return rc;
   if ((rc = m->rope.ensure(t * (d.head_dim / 2) * sizeof(float2)))) return rc;
@@ -365,9 +405,8 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   std::vector<int32_t> ctx(B);
   for (int i = 0; i < B; ++i) ctx[i] = kv->ctx_len[seq_ids[i]];
   std::vector<AttnItem> items;
-  std::vector<AttnMerge> merges;
   int n_slots = 0;
-  build_attention_work(m, B, lens, ctx.data(), items, merges, &n_slots);
+  build_attention_work(m, B, lens, ctx.data(), items, &n_slots);
 
   BatchLayout L;
   L.B = B;
@@ -381,10 +420,8 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   L.off_tseq = take(T);
   L.off_tok = take(tokens_on_device ? 0 : T);
   L.off_items = take(items.size() * 8);
-  L.off_merges = take(merges.size() * 8);
   L.total = o;
   L.n_items = static_cast<int>(items.size());
-  L.n_merges = static_cast<int>(merges.size());
   L.n_slots = n_slots;
 
   int rc;
@@ -392,6 +429,8 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   const int hd = m->d.head_dim;
   if ((rc = m->attn_part_o.ensure(static_cast<size_t>(std::max(1, n_slots)) * 128 * hd * 4))) return rc;
   if ((rc = m->attn_part_ml.ensure(static_cast<size_t>(std::max(1, n_slots)) * 128 * 2 * 4))) return rc;
+  // One counter per split query tile; every launch leaves them at zero again.
+  if ((rc = m->attn_counters.ensure(static_cast<size_t>(std::max(1, n_slots)) * 4, true))) return rc;
   if ((rc = m->stg.dev.ensure(L.total * 4))) return rc;
   int slot;
   if ((rc = staging_slot(m->stg, L.total, &slot))) return rc;
@@ -409,7 +448,6 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   }
   if (!tokens_on_device) std::memcpy(h + L.off_tok, tokens, sizeof(int32_t) * T);
   if (!items.empty()) std::memcpy(h + L.off_items, items.data(), items.size() * sizeof(AttnItem));
-  if (!merges.empty()) std::memcpy(h + L.off_merges, merges.data(), merges.size() * sizeof(AttnMerge));
   CS_CUDA(cudaMemcpyAsync(m->stg.dev.p, h, L.total * 4, cudaMemcpyHostToDevice, s));
   CS_CUDA(cudaEventRecord(m->stg.ev[slot], s));
   m->stg.pending[slot] = true;
@@ -554,7 +592,7 @@ int cs_model_free(cs_model* m) {
   cudaDeviceSynchronize();
   for (void* p : m->owned) cudaFree(p);
   DevBuf* bufs[] = {&m->x, &m->a, &m->qkv, &m->attn_o, &m->hmlp, &m->rope, &m->h_last, &m->lm_part, &m->vlogits,
-                    &m->logits, &m->lse, &m->attn_part_o, &m->attn_part_ml, &m->stg.dev};
+                    &m->logits, &m->lse, &m->attn_part_o, &m->attn_part_ml, &m->attn_counters, &m->stg.dev};
   for (DevBuf* b : bufs) b->release();
   for (cudaEvent_t e : m->prof.pool) cudaEventDestroy(e);
   for (int i = 0; i < kStagingRing; ++i) {
@@ -614,7 +652,7 @@ int cs_kv_alloc(const cs_model* m, int num_pages, int page_size, int max_seqs, i
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&kv->upload_ev, cudaEventDisableTiming);
   if (e != cudaSuccess) { rc = cuda_fail(e, "kv page table"); cs_kv_free(kv); return rc; }
   std::memset(kv->table_host, 0, tbytes);
-  if (!make_tensor_map_16b(&kv->tm_pool, kv->pool, rows, m->d.head_dim, kPageSize, 64, true, true)) {
+  if (!make_kv_group_map(&kv->tm_pool, kv->pool, rows, m->d.head_dim, kPageSize / 8)) {
     g_cuda_error = "cuTensorMapEncodeTiled failed for the kv pool";
     cs_kv_free(kv);
     return CS_ECUDA;

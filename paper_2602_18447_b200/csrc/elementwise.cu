@@ -99,10 +99,13 @@ __global__ void kv_scatter_kernel(const uint16_t* __restrict__ src_k, const uint
   const size_t src = static_cast<size_t>(t) * row_stride + c * 8;
   uint4 k = *reinterpret_cast<const uint4*>(src_k + src);
   uint4 v = *reinterpret_cast<const uint4*>(src_v + src);
-  if (src_is_f16) {  // the cache format is bf16: round the fp16 activations
+  if (src_is_f16) {  // the cache keeps bf16 precision: round the fp16 activations to the nearest bf16 value
     k = make_uint4(f16x2_to_bf16x2(k.x), f16x2_to_bf16x2(k.y), f16x2_to_bf16x2(k.z), f16x2_to_bf16x2(k.w));
     v = make_uint4(f16x2_to_bf16x2(v.x), f16x2_to_bf16x2(v.y), f16x2_to_bf16x2(v.z), f16x2_to_bf16x2(v.w));
   }
+  // ... and stores those bf16 values in the fp16 encoding, the operand format of the attention products
+  k = make_uint4(bf16x2_to_f16x2(k.x), bf16x2_to_f16x2(k.y), bf16x2_to_f16x2(k.z), bf16x2_to_f16x2(k.w));
+  v = make_uint4(bf16x2_to_f16x2(v.x), bf16x2_to_f16x2(v.y), bf16x2_to_f16x2(v.z), bf16x2_to_f16x2(v.w));
   *reinterpret_cast<uint4*>(pool_k + dst) = k;
   *reinterpret_cast<uint4*>(pool_v + dst) = v;
 }

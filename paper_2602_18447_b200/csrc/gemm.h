@@ -22,6 +22,18 @@ bool make_tensor_map_16b(CUtensorMap* tm, const void* base, uint64_t rows, uint6
 // (token, head-in-group) pairs.
 bool make_tensor_map_heads3d(CUtensorMap* tm, const void* base, uint64_t tokens, uint64_t heads, uint32_t head_dim,
                              uint64_t row_elems, uint32_t box_tokens, uint32_t box_heads);
+// 4D fp16 tensor maps that deliver rows of `hd` columns (hd = 64 * halves) as
+// [8-row group][64-column half][8 rows][128 bytes] with the 128-byte swizzle, the shared-memory layout of the
+// attention kernel's K and V tiles. Dimensions, innermost first: 64 columns, 8 rows (stride = one row), halves
+// (stride 128 bytes), groups.
+//  - make_kv_group_map: over a matrix of `rows` rows (a multiple of 8) of exactly hd columns; the last coordinate
+//    is the 8-row group index; one box = groups_per_box groups. Used for the cache pool (one 16-row page per box).
+//  - make_kv_rows_map: over a row-major [rows_alloc, row_elems] matrix whose rows hold many 64-column blocks; the
+//    second coordinate is the first row (any value < rows), the third the 64-column block index, the last is
+//    always 0 and spans 16 groups, so one box = 128 consecutive rows starting at any row. The box may reach up to
+//    127 rows past `rows`: the allocation must hold them (rows_alloc >= rows + 128) and they must be finite.
+bool make_kv_group_map(CUtensorMap* tm, const void* base, uint64_t rows, uint32_t hd, uint32_t groups_per_box);
+bool make_kv_rows_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t row_elems, uint32_t hd);
 // Tensor map of a GEMM operand ([rows, k] fp16, K-major): 128-row x 64-column boxes, 128-byte swizzle.
 bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k);
 

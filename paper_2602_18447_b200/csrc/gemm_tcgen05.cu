@@ -334,6 +334,33 @@ bool make_tensor_map_heads3d(CUtensorMap* tm, const void* base, uint64_t tokens,
   return r == CUDA_SUCCESS;
 }
 
+bool make_kv_group_map(CUtensorMap* tm, const void* base, uint64_t rows, uint32_t hd, uint32_t groups_per_box) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || hd % 64 || rows % 8) return false;
+  cuuint64_t dims[4] = {64, 8, hd / 64, rows / 8};
+  cuuint64_t strides[3] = {static_cast<cuuint64_t>(hd) * 2, 128, static_cast<cuuint64_t>(hd) * 2 * 8};
+  cuuint32_t box[4] = {64, 8, hd / 64, groups_per_box};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+bool make_kv_rows_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t row_elems, uint32_t hd) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || hd % 64 || row_elems % 64) return false;
+  // The row coordinate (dimension 1) and the group coordinate (dimension 3) address the same rows: row + 8 * group.
+  cuuint64_t dims[4] = {64, rows + 8, row_elems / 64, 16};
+  cuuint64_t strides[3] = {row_elems * 2, 128, row_elems * 2 * 8};
+  cuuint32_t box[4] = {64, 8, hd / 64, 16};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k) {
   return make_tensor_map_16b(tm, base, static_cast<uint64_t>(rows), static_cast<uint64_t>(k), 128, 64, true, false);
 }

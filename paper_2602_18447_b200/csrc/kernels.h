@@ -10,22 +10,19 @@ namespace cs {
 constexpr int kNumSMs = 148;
 
 // One unit of attention work: the query rows of 128 / G consecutive new tokens of one step for the G query
-// heads of one kv head (row = token * G + head-in-group, at most 128 rows), over a range of 64-key tiles.
-// Key tiles 0 .. ctx_tiles-1 cover the cached context (4 pages each), the following ones the step's own
-// new keys.
+// heads of one kv head (row = token * G + head-in-group, at most 128 rows), over a range of 128-key tiles.
+// Key tiles 0 .. ctx_tiles-1 cover the cached context (8 pages each), the following ones the step's own
+// new keys. A query tile whose key range is cut into n_splits > 1 pieces owns the partial-result slots
+// [slot0, slot0 + n_splits) and the counter counters[slot0].
 struct AttnItem {
   int32_t step;       // index into the batch
   int32_t kv_head;
   int32_t q_tok0;     // first new token of the query tile, relative to the step (multiple of 128 / G)
   int32_t tile_begin; // key tile range [tile_begin, tile_end)
   int32_t tile_end;
-  int32_t slot;       // partial-result slot, or -1 when the range is the whole key sequence
-  int32_t pad0, pad1;
-};
-
-// A group of partial results to merge: slots [slot0, slot0 + n_splits) belong to one query tile.
-struct AttnMerge {
-  int32_t step, kv_head, q_tok0, slot0, n_splits, pad0, pad1, pad2;
+  int32_t slot;       // this piece's partial-result slot (unused when n_splits == 1)
+  int32_t slot0;      // first slot of the query tile
+  int32_t n_splits;   // pieces the query tile's key range is cut into (1 = whole range, at most 32)
 };
 
 struct AttnParams {
@@ -37,10 +34,11 @@ struct AttnParams {
   const int32_t* page_table;// [max_seqs, max_pages_per_seq]
   int32_t max_pages_per_seq;
   int32_t n_q_heads, n_kv_heads, head_dim, n_qkv;
-  int32_t k_row_base, v_row_base;  // first pool row of this layer's K and V planes
+  int32_t k_group_base, v_group_base;  // first 8-row group of this layer's K and V planes in the pool
   float scale_log2e;        // log2(e) / sqrt(head_dim)
   float* part_o;            // [slots, 128, hd] unnormalised partial outputs
   float* part_ml;           // [slots, 128, 2]  exponent reference (raw score units) and sum
+  int32_t* counters;        // [slots] zero between launches
   uint32_t* status;
 };
 
@@ -56,7 +54,8 @@ cudaError_t launch_rope_apply(uint16_t* qkv, const float2* table, int T, int n_q
                               cudaStream_t s);
 // Copy K and V rows into cache pages. src rows are [n_kv_heads*hd] wide at src_k/src_v + t*row_stride.
 // Row t goes to sequence tok_seq[t], position tok_pos[t]; when tok_seq is NULL, to sequence const_seq,
-// position pos0 + t.
+// position pos0 + t. The cache holds bf16 values in the fp16 encoding: bf16 sources are re-encoded (exact in
+// the fp16 normal range), fp16 sources are first rounded to the nearest bf16 value.
 cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int row_stride, const int32_t* tok_seq,
                               const int32_t* tok_pos, int const_seq, int pos0, const int32_t* page_table,
                               int max_pages_per_seq,
@@ -65,11 +64,12 @@ cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int 
 // Re-encode n bf16 values (n even) as fp16 in place.
 cudaError_t launch_bf16_to_f16(uint16_t* p, size_t n, cudaStream_t s);
 
-// tm_pool: 2D map of the bf16 cache (16-row x 64-column boxes); tm_qkv: 2D map of the fp16 qkv workspace with
-// the same box; tm_q3d: 3D map (head_dim, head, token) of the same workspace with box (64, G, 128 / G).
-cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_pool, const CUtensorMap& tm_qkv,
-                             const CUtensorMap& tm_q3d, const AttnItem* items, int n_items, const AttnMerge* merges,
-                             int n_merges, cudaStream_t s);
+// tm_pool: 4D map of the cache (make_kv_group_map over all pool rows, one 16-row page per box); tm_kv_new: the
+// same kind of map over the qkv workspace (128 rows per box; see make_kv_rows_map); tm_q3d: 3D map (head_dim,
+// head, token) of the workspace with box (64, G, 128 / G).
+cudaError_t launch_attention(const AttnParams& p, const CUtensorMap& tm_pool, const CUtensorMap& tm_kv_new,
+                             const CUtensorMap& tm_q3d, const AttnItem* items, int n_items, cudaStream_t s);
+int attention_max_splits();
 
 // h[b] = RMSNorm(x[last_row[b]]) as bf16 [B_pad, d]; rows B..B_pad-1 are zeroed.
 cudaError_t launch_last_rows_norm(const float* x, const int32_t* cu_new, const float* gain, uint16_t* h, int B,
