@@ -153,7 +153,7 @@ int staging_slot(Staging& st, size_t ints, int* slot_out) {
 
 struct BatchLayout {
   int B = 0, T = 0;
-  size_t off_cu, off_ctx, off_seq, off_pos, off_tseq, off_tok, off_items, total;
+  size_t off_cu, off_pos, off_tseq, off_tok, off_items, total;
   int n_items = 0, n_slots = 0;
 };
 
@@ -230,7 +230,8 @@ void build_attention_work(const cs_model* m, int B, const int32_t* lens, const i
       for (int s = 0; s < n; ++s) {
         const int b = static_cast<int>(static_cast<long>(u.nt) * s / n);
         const int e = static_cast<int>(static_cast<long>(u.nt) * (s + 1) / n);
-        items.push_back(AttnItem{u.step, h, u.q0, b, e, n > 1 ? slots + s : 0, n > 1 ? slots : 0, n});
+        items.push_back(AttnItem{u.step, h, u.q0, b, e, n > 1 ? slots + s : 0, n > 1 ? slots : 0, n, 0, lens[u.step],
+                                 ctx[u.step], 0, {0, 0, 0, 0}});
       }
       if (n > 1) slots += n;
     }
@@ -295,9 +296,6 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
                const int32_t* d_tok, cudaStream_t s) {
   const cs_model_desc& d = m->d;
   const int T = L.T;
-  const int32_t* d_cu = dev_meta + L.off_cu;
-  const int32_t* d_ctx = dev_meta + L.off_ctx;
-  const int32_t* d_seq = dev_meta + L.off_seq;
   const int32_t* d_pos = dev_meta + L.off_pos;
   const int32_t* d_tseq = dev_meta + L.off_tseq;
   const AttnItem* d_items = reinterpret_cast<const AttnItem*>(dev_meta + L.off_items);
@@ -326,9 +324,6 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   AttnParams ap;
   ap.qkv = qkv;
   ap.out = attn_o;
-  ap.cu_new = d_cu;
-  ap.ctx_len = d_ctx;
-  ap.seq_id = d_seq;
   ap.page_table = kv->table_dev;
   ap.max_pages_per_seq = kv->max_pages_per_seq;
   ap.n_q_heads = d.n_q_heads;
@@ -414,12 +409,10 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   size_t o = 0;
   auto take = [&o](size_t n) { size_t r = o; o += (n + 3) & ~size_t(3); return r; };  // keep 16-byte alignment
   L.off_cu = take(B + 1);
-  L.off_ctx = take(B);
-  L.off_seq = take(B);
   L.off_pos = take(T);
   L.off_tseq = take(T);
   L.off_tok = take(tokens_on_device ? 0 : T);
-  L.off_items = take(items.size() * 8);
+  L.off_items = take(items.size() * (sizeof(AttnItem) / 4));
   L.total = o;
   L.n_items = static_cast<int>(items.size());
   L.n_slots = n_slots;
@@ -439,14 +432,16 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   cu[0] = 0;
   for (int i = 0; i < B; ++i) {
     cu[i + 1] = cu[i] + lens[i];
-    h[L.off_ctx + i] = ctx[i];
-    h[L.off_seq + i] = seq_ids[i];
     for (int p = 0; p < lens[i]; ++p) {
       h[L.off_pos + cu[i] + p] = ctx[i] + p;
       h[L.off_tseq + cu[i] + p] = seq_ids[i];
     }
   }
   if (!tokens_on_device) std::memcpy(h + L.off_tok, tokens, sizeof(int32_t) * T);
+  for (AttnItem& it : items) {
+    it.tok0 = cu[it.step];
+    it.seq = seq_ids[it.step];
+  }
   if (!items.empty()) std::memcpy(h + L.off_items, items.data(), items.size() * sizeof(AttnItem));
   CS_CUDA(cudaMemcpyAsync(m->stg.dev.p, h, L.total * 4, cudaMemcpyHostToDevice, s));
   CS_CUDA(cudaEventRecord(m->stg.ev[slot], s));

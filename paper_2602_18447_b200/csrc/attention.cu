@@ -4,13 +4,16 @@
 // of one kv head (ntok = 128 / G, so at most 128 rows = the 128 lanes of the tensor memory; row = token * G +
 // head-in-group), and a range of 128-key tiles. Context keys are all visible; the step's own keys are causal.
 //
-//   warp 0        TMA producer. Q tile once; then, per key tile, K into a ring of K stages and V into a ring
-//                 of V stages. A cached tile is 8 pages, one 4D box per page, issued by 8 lanes at once; a tile
-//                 of the step's own keys is one box from the qkv workspace. Every box lands as
-//                 [8-key group][64-column half][8 keys][128 B] with the 128-byte swizzle, which serves K as a
-//                 K-major operand and V as an MN-major operand with uniform strides.
-//   warp 1        one thread issues tcgen05.mma: S_j = Q K_j^T into one of two TMEM buffers (both operands from
-//                 shared memory), O += P_j V_j with P_j read from TMEM.
+//   warp 0        TMA producer of Q (once) and of the K tiles, into a ring of K stages
+//   warp 6        TMA producer of the V tiles, into a ring of V stages
+//                 A cached tile is 8 pages, one 4D box per page, issued by 8 lanes at once (one thread issuing
+//                 them in turn takes about three times as long); a tile of the step's own keys is one box from
+//                 the qkv workspace. Every box lands as [8-key group][64-column half][8 keys][128 B] with the
+//                 128-byte swizzle, which serves K as a K-major operand and V as an MN-major operand with
+//                 uniform strides.
+//   warp 1        one thread issues tcgen05.mma: S_j = Q K_j^T into one of three TMEM buffers (both operands from
+//                 shared memory), O += P_j V_j with P_j read from TMEM. S_{j+2} is issued before P_j V_j, so the
+//                 softmax never waits for the tensor core.
 //   warps 2..5    softmax: one thread per query row reads its S row from TMEM, keeps the running reference
 //                 maximum and the sum in registers and writes P_j (fp16) back into the columns S_j came from.
 //
@@ -30,10 +33,11 @@ namespace {
 constexpr int kKTile = 128;
 constexpr int kPage = 16;
 constexpr int kPagesPerTile = kKTile / kPage;
-constexpr int kAttnThreads = 192;
+constexpr int kAttnThreads = 224;
 constexpr int kStages = 3;                  // K stages and, separately, V stages
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 constexpr int kMaxSplits = 32;
+constexpr int kSBufs = 3;                   // S/P buffers in tensor memory
 
 template <int HD>
 struct AttnSmem {
@@ -49,8 +53,8 @@ struct AttnSmem {
   static constexpr int kUsed = kBarOff + 256 + 1024;                   // + slack for 1024-byte alignment
   // At least 116 KB so that two CTAs never share an SM: each allocates all 512 TMEM columns.
   static constexpr int kTotal = kUsed > 118784 ? kUsed : 118784;
-  static constexpr uint32_t kTmemCols = 512;                           // S0 [0,128), S1 [128,256), O [256,256+HD)
-  static constexpr uint32_t kOCol = 256;
+  static constexpr uint32_t kTmemCols = 512;                           // S0, S1, S2 at 0, 128, 256; O [384,384+HD)
+  static constexpr uint32_t kOCol = 384;
 };
 
 // Shared-memory descriptor, 128-byte swizzle: `lbo` = distance between 64-element blocks along the contiguous
@@ -68,15 +72,146 @@ __host__ __device__ constexpr uint32_t idesc_f16(int m, int n, bool b_mn_major) 
   return (1u << 4) | (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
          (static_cast<uint32_t>(m >> 4) << 24);
 }
-// D[tmem] (+)= A[tmem] * B[smem]: A is 128 lanes x 16 fp16 values, two per 32-bit column.
-__device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accumulate) {
+// The thread that feeds the tensor core must not stall: even a wait on a barrier that is already complete costs a
+// round trip of a few hundred cycles, in which the short queue of issued products runs dry. Both groups below
+// therefore start with a non-blocking test of the barrier the NEXT group will need, issue their products and
+// their two completion arrivals, and only then read the test's answer (true = that phase is complete).
+
+// S = Q K^T for one 128-key tile: HD / 16 products with both operands in shared memory. The Q tile is
+// [half][128 rows][128 B]; the K tile [8-key group][half][8 keys][128 B].
+template <int HD>
+__device__ __forceinline__ bool umma_qk_group(uint32_t tmem_s, uint64_t q_desc, uint64_t k_desc, uint32_t idesc,
+                                              uint64_t* commit1, uint64_t* commit2, uint64_t* peek_bar,
+                                              uint32_t peek_parity);
+template <>
+__device__ __forceinline__ bool umma_qk_group<128>(uint32_t tmem_s, uint64_t q_desc, uint64_t k_desc, uint32_t idesc,
+                                                   uint64_t* commit1, uint64_t* commit2, uint64_t* peek_bar,
+                                                   uint32_t peek_parity) {
+  uint32_t ready;
   asm volatile(
-      "{\n\t.reg .pred P;\n\t"
-      "setp.ne.b32 P, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, P;\n\t}"
-      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred P;\n\t.reg .b64 da, db;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, 0;\n\t"
+      "add.u64 da, %4, 2;\n\tadd.u64 db, %5, 2;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "add.u64 da, %4, 4;\n\tadd.u64 db, %5, 4;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "add.u64 da, %4, 6;\n\tadd.u64 db, %5, 6;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "add.u64 da, %4, 1024;\n\tadd.u64 db, %5, 64;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "add.u64 da, %4, 1026;\n\tadd.u64 db, %5, 66;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "add.u64 da, %4, 1028;\n\tadd.u64 db, %5, 68;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "add.u64 da, %4, 1030;\n\tadd.u64 db, %5, 70;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%7];\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ready)
+      : "r"(smem_u32(peek_bar)), "r"(peek_parity), "r"(tmem_s), "l"(q_desc), "l"(k_desc), "r"(idesc),
+        "r"(smem_u32(commit1)), "r"(smem_u32(commit2))
       : "memory");
+  return ready != 0;
+}
+template <>
+__device__ __forceinline__ bool umma_qk_group<64>(uint32_t tmem_s, uint64_t q_desc, uint64_t k_desc, uint32_t idesc,
+                                                  uint64_t* commit1, uint64_t* commit2, uint64_t* peek_bar,
+                                                  uint32_t peek_parity) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t.reg .b64 da, db;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, 0;\n\t"
+      "add.u64 da, %4, 2;\n\tadd.u64 db, %5, 2;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "add.u64 da, %4, 4;\n\tadd.u64 db, %5, 4;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "add.u64 da, %4, 6;\n\tadd.u64 db, %5, 6;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, 1;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%7];\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ready)
+      : "r"(smem_u32(peek_bar)), "r"(peek_parity), "r"(tmem_s), "l"(q_desc), "l"(k_desc), "r"(idesc),
+        "r"(smem_u32(commit1)), "r"(smem_u32(commit2))
+      : "memory");
+  return ready != 0;
+}
+
+// O (+)= P V for one 128-key tile: eight products of 16 keys each. P comes from tensor memory (128 lanes x 16 fp16
+// values per product, two per 32-bit column, so 8 columns per product); V from shared memory, one 16-key page per
+// product.
+template <int HD>
+__device__ __forceinline__ bool umma_pv_group(uint32_t tmem_o, uint32_t tmem_p, uint64_t v_desc, uint32_t idesc,
+                                              uint32_t accumulate_first, uint64_t* commit1, uint64_t* commit2,
+                                              uint64_t* peek_bar, uint32_t peek_parity);
+template <>
+__device__ __forceinline__ bool umma_pv_group<128>(uint32_t tmem_o, uint32_t tmem_p, uint64_t v_desc, uint32_t idesc,
+                                                   uint32_t accumulate_first, uint64_t* commit1, uint64_t* commit2,
+                                                   uint64_t* peek_bar, uint32_t peek_parity) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred P, Q;\n\t.reg .b64 db;\n\t.reg .b32 ta;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "setp.ne.b32 Q, %7, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [%4], %5, %6, Q;\n\t"
+      "add.u32 ta, %4, 8;\n\tadd.u64 db, %5, 256;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 16;\n\tadd.u64 db, %5, 512;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 24;\n\tadd.u64 db, %5, 768;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 32;\n\tadd.u64 db, %5, 1024;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 40;\n\tadd.u64 db, %5, 1280;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 48;\n\tadd.u64 db, %5, 1536;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 56;\n\tadd.u64 db, %5, 1792;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ready)
+      : "r"(smem_u32(peek_bar)), "r"(peek_parity), "r"(tmem_o), "r"(tmem_p), "l"(v_desc), "r"(idesc),
+        "r"(accumulate_first), "r"(smem_u32(commit1)), "r"(smem_u32(commit2))
+      : "memory");
+  return ready != 0;
+}
+template <>
+__device__ __forceinline__ bool umma_pv_group<64>(uint32_t tmem_o, uint32_t tmem_p, uint64_t v_desc, uint32_t idesc,
+                                                  uint32_t accumulate_first, uint64_t* commit1, uint64_t* commit2,
+                                                  uint64_t* peek_bar, uint32_t peek_parity) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred P, Q;\n\t.reg .b64 db;\n\t.reg .b32 ta;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "setp.ne.b32 Q, %7, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [%4], %5, %6, Q;\n\t"
+      "add.u32 ta, %4, 8;\n\tadd.u64 db, %5, 128;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 16;\n\tadd.u64 db, %5, 256;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 24;\n\tadd.u64 db, %5, 384;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 32;\n\tadd.u64 db, %5, 512;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 40;\n\tadd.u64 db, %5, 640;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 48;\n\tadd.u64 db, %5, 768;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "add.u32 ta, %4, 56;\n\tadd.u64 db, %5, 896;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], [ta], db, %6, 1;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ready)
+      : "r"(smem_u32(peek_bar)), "r"(peek_parity), "r"(tmem_o), "r"(tmem_p), "l"(v_desc), "r"(idesc),
+        "r"(accumulate_first), "r"(smem_u32(commit1)), "r"(smem_u32(commit2))
+      : "memory");
+  return ready != 0;
 }
 
 __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -118,9 +253,9 @@ struct Bars {
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages];   // TMA landed / Q K^T of the tile complete
   uint64_t v_full[kStages], v_empty[kStages];   // TMA landed / P V of the tile complete
-  uint64_t s_full[2];                           // Q K^T complete
-  uint64_t p_full[2];                           // P written by the 4 softmax warps
-  uint64_t pv_done[2];                          // P V complete
+  uint64_t s_full[kSBufs];                      // Q K^T complete
+  uint64_t p_full[kSBufs];                      // P written by the 4 softmax warps
+  uint64_t pv_done[kSBufs];                     // P V complete
   uint32_t tmem_slot;
   uint32_t abort_flag;
   uint32_t is_last;
@@ -139,9 +274,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
 
   const AttnItem it = items[blockIdx.x];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tok0 = p.cu_new[it.step];
-  const int n_new = p.cu_new[it.step + 1] - tok0;
-  const int ctx = p.ctx_len[it.step];
+  const int tok0 = it.tok0, n_new = it.n_new, ctx = it.ctx;
   const int G = p.n_q_heads / p.n_kv_heads;
   const int ctx_tiles = (ctx + kKTile - 1) / kKTile;
   const int n_tiles = it.tile_end - it.tile_begin;
@@ -154,7 +287,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       mbar_init(&bars->v_full[s], 1);
       mbar_init(&bars->v_empty[s], 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < kSBufs; ++b) {
       mbar_init(&bars->s_full[b], 1);
       mbar_init(&bars->p_full[b], 4);
       mbar_init(&bars->pv_done[b], 1);
@@ -170,20 +303,32 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
     tmem_alloc(&bars->tmem_slot, L::kTmemCols);
     tmem_relinquish();
   }
+  {
+    // The Q box covers (128 / G) * G rows; the rest of the 128-row operand is zeroed so that its scores are finite.
+    // A row keeps to its own 128 bytes under the swizzle.
+    const int used_rows = (128 / G) * G;
+    const int n16 = (128 - used_rows) * 8;
+    for (int i = threadIdx.x; i < n16 * L::kHalves; i += kAttnThreads) {
+      const int h = i / n16, r = i - h * n16;
+      reinterpret_cast<uint4*>(smem + L::kQOff + h * 128 * 128 + used_rows * 128)[r] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    fence_proxy_async();
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_slot;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer (whole warp)
-    if (lane == 0) {
+  if (warp == 0 || warp == 6) {
+    // ------------------------------------------------------------ TMA producers (whole warps): warp 0 K, warp 6 V
+    const bool is_k = warp == 0;
+    if (is_k && lane == 0) {
       mbar_arrive_expect_tx(&bars->q_full, L::kHalves * (128 / G) * G * 128);
 #pragma unroll
       for (int h = 0; h < L::kHalves; ++h)
         tma_load_3d(smem + L::kQOff + h * 128 * 128, &tm_q3d, &bars->q_full, h * 64, it.kv_head * G, tok0 + it.q_tok0);
     }
-    const int32_t* pages = p.page_table + static_cast<size_t>(p.seq_id[it.step]) * p.max_pages_per_seq;
+    const int32_t* pages = p.page_table + static_cast<size_t>(it.seq) * p.max_pages_per_seq;
     const int n_pages = (ctx + kPage - 1) / kPage;
     // Lane l < 8 fetches page l of a cached tile. Pages past the end of the context are replaced by the last
     // real page; their keys are masked.
@@ -191,43 +336,30 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       return (t < ctx_tiles && lane < kPagesPerTile) ? __ldg(pages + min(t * kPagesPerTile + lane, n_pages - 1)) : 0;
     };
     int page = page_of(it.tile_begin);
-    const int kcol = (p.n_q_heads + it.kv_head) * L::kHalves;                  // in 64-column units
-    const int vcol = (p.n_q_heads + p.n_kv_heads + it.kv_head) * L::kHalves;
+    // column of this kv head's K (or V) in the qkv workspace, in 64-column units
+    const int col = (p.n_q_heads + (is_k ? 0 : p.n_kv_heads) + it.kv_head) * L::kHalves;
+    const int group_base = is_k ? p.k_group_base : p.v_group_base;
+    uint64_t* full = is_k ? bars->k_full : bars->v_full;
+    uint64_t* empty = is_k ? bars->k_empty : bars->v_empty;
+    uint8_t* ring = smem + (is_k ? L::kKOff : L::kVOff);
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     for (int t = it.tile_begin; t < it.tile_end; ++t) {
       const int next_page = page_of(t + 1 < it.tile_end ? t + 1 : t);
-      const bool cached = t < ctx_tiles;
       const int group = ((page * p.n_kv_heads + it.kv_head) * kPage) >> 3;     // 8-row group within a K or V plane
-      const int row0 = tok0 + (t - ctx_tiles) * kKTile;                        // first own-key row of a new tile
-      uint8_t* sk = smem + L::kKOff + stage * L::kTileBytes;
-      uint8_t* sv = smem + L::kVOff + stage * L::kTileBytes;
-      // ---- K
-      if (lane == 0) ok = mbar_wait(&bars->k_empty[stage], phase ^ 1u, abort_flag, p.status);
+      uint8_t* dst = ring + stage * L::kTileBytes;
+      if (lane == 0) ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      if (lane == 0) mbar_arrive_expect_tx(&bars->k_full[stage], L::kTileBytes);
+      if (lane == 0) mbar_arrive_expect_tx(&full[stage], L::kTileBytes);
       __syncwarp();
-      if (cached) {
-        if (lane < kPagesPerTile)
-          tma_load_4d(sk + lane * L::kPageBytes, &tm_pool, &bars->k_full[stage], 0, 0, 0, p.k_group_base + group);
+      if (t < ctx_tiles) {
+        if (lane < kPagesPerTile) tma_load_4d(dst + lane * L::kPageBytes, &tm_pool, &full[stage], 0, 0, 0, group_base + group);
       } else if (lane == 0) {
         // Rows past the step's own tokens belong to the next step or to the zeroed tail of the workspace;
         // their keys are masked.
-        tma_load_4d(sk, &tm_kv_new, &bars->k_full[stage], 0, row0, kcol, 0);
-      }
-      // ---- V
-      if (lane == 0) ok = mbar_wait(&bars->v_empty[stage], phase ^ 1u, abort_flag, p.status);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if (lane == 0) mbar_arrive_expect_tx(&bars->v_full[stage], L::kTileBytes);
-      __syncwarp();
-      if (cached) {
-        if (lane < kPagesPerTile)
-          tma_load_4d(sv + lane * L::kPageBytes, &tm_pool, &bars->v_full[stage], 0, 0, 0, p.v_group_base + group);
-      } else if (lane == 0) {
-        tma_load_4d(sv, &tm_kv_new, &bars->v_full[stage], 0, row0, vcol, 0);
+        tma_load_4d(dst, &tm_kv_new, &full[stage], 0, tok0 + (t - ctx_tiles) * kKTile, col, 0);
       }
       page = next_page;
       if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -241,42 +373,39 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
     if (lane == 0) {
       constexpr uint32_t kIdescQK = idesc_f16(128, kKTile, false);
       constexpr uint32_t kIdescPV = idesc_f16(128, HD, true);
-      const uint32_t q_addr = smem_u32(smem + L::kQOff);
+      const uint64_t q_desc = smem_desc(smem_u32(smem + L::kQOff), 16, 1024);
+      const uint64_t k_desc0 = smem_desc(smem_u32(smem + L::kKOff), 16, L::kGroupBytes);
+      const uint64_t v_desc0 = smem_desc(smem_u32(smem + L::kVOff), 1024, L::kGroupBytes);
       bool ok = mbar_wait(&bars->q_full, 0, abort_flag, p.status);
       int k_stage = 0, v_stage = 0;
       uint32_t k_phase = 0, v_phase = 0;
-      for (int j = 0; j <= n_tiles && ok; ++j) {
-        if (j < n_tiles) {
-          // S_b is free: P V of tile j-2, which read P from these columns, was issued before this product.
-          const int b = j & 1;
-          if (!mbar_wait(&bars->k_full[k_stage], k_phase, abort_flag, p.status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t k_addr = smem_u32(smem + L::kKOff + k_stage * L::kTileBytes);
-#pragma unroll
-          for (int k = 0; k < HD / 16; ++k) {
-            const uint64_t adesc = smem_desc(q_addr + (k >> 2) * (128 * 128) + (k & 3) * 32, 16, 1024);
-            const uint64_t bdesc = smem_desc(k_addr + (k >> 2) * 1024 + (k & 3) * 32, 16, L::kGroupBytes);
-            umma_f16(tmem_base + b * kKTile, adesc, bdesc, kIdescQK, k != 0);
-          }
-          umma_commit(&bars->s_full[b]);
-          umma_commit(&bars->k_empty[k_stage]);
+      bool k_ready = false, v_ready = false;
+      // Issue order: S_0, S_1, then for every tile j: S_{j+2}, O += P_j V_j. With three S/P buffers S_{j+2} lands in the
+      // buffer that P_{j-1} V_{j-1} (issued earlier, and executed in issue order) has read P from, while the softmax
+      // works on S_j and S_{j+1} waits in the third: the softmax never waits for the tensor core.
+      for (int j = -2; j < n_tiles && ok; ++j) {
+        if (j + 2 < n_tiles) {
+          const int b = (j + 2) % kSBufs;
+          if (!k_ready && !mbar_wait(&bars->k_full[k_stage], k_phase, abort_flag, p.status)) { ok = false; break; }
+          // next needed: V of tile j (or of tile 0)
+          v_ready = umma_qk_group<HD>(tmem_base + b * kKTile, q_desc,
+                                      k_desc0 + static_cast<uint64_t>(k_stage * (L::kTileBytes >> 4)), kIdescQK,
+                                      &bars->s_full[b], &bars->k_empty[k_stage], &bars->v_full[v_stage], v_phase);
           if (++k_stage == kStages) { k_stage = 0; k_phase ^= 1u; }
+          k_ready = false;
         }
-        if (j > 0) {
-          const int i = j - 1, b = i & 1;
-          const uint32_t use = static_cast<uint32_t>(i >> 1) & 1u;
-          if (!mbar_wait(&bars->v_full[v_stage], v_phase, abort_flag, p.status) ||
+        if (j >= 0) {
+          const int b = j % kSBufs;
+          const uint32_t use = static_cast<uint32_t>(j / kSBufs) & 1u;
+          if ((!v_ready && !mbar_wait(&bars->v_full[v_stage], v_phase, abort_flag, p.status)) ||
               !mbar_wait(&bars->p_full[b], use, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t v_addr = smem_u32(smem + L::kVOff + v_stage * L::kTileBytes);
-#pragma unroll
-          for (int ks = 0; ks < kKTile / 16; ++ks) {
-            const uint64_t bdesc = smem_desc(v_addr + ks * L::kPageBytes, 1024, L::kGroupBytes);
-            umma_f16_ts(tmem_base + L::kOCol, tmem_base + b * kKTile + ks * 8, bdesc, kIdescPV, (i | ks) != 0);
-          }
-          umma_commit(&bars->v_empty[v_stage]);
-          umma_commit(&bars->pv_done[b]);
+          // next needed: K of tile j+3
+          k_ready = umma_pv_group<HD>(tmem_base + L::kOCol, tmem_base + b * kKTile,
+                                      v_desc0 + static_cast<uint64_t>(v_stage * (L::kTileBytes >> 4)), kIdescPV, j != 0,
+                                      &bars->v_empty[v_stage], &bars->pv_done[b], &bars->k_full[k_stage], k_phase);
           if (++v_stage == kStages) { v_stage = 0; v_phase ^= 1u; }
+          v_ready = false;
         }
       }
     }
@@ -291,14 +420,16 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
     const bool row_ok = (p_local < ntok) && (pos < n_new);
     const float sc = p.scale_log2e;
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-    float m_ref = -INFINITY;   // raw score units
+    // Reference of the exponents, raw score units; -inf until the row meets a visible key. Unused rows of the tile
+    // start at 0 so that they never ask for the first-sight maximum.
+    float m_ref = row_ok ? -INFINITY : 0.f;
     float l = 0.f;
     bool ok = true;
 
     for (int j = 0; j < n_tiles; ++j) {
       const int t = it.tile_begin + j;
-      const int b = j & 1;
-      const uint32_t use = static_cast<uint32_t>(j >> 1) & 1u;
+      const int b = j % kSBufs;
+      const uint32_t use = static_cast<uint32_t>(j / kSBufs) & 1u;
       if (!mbar_wait(&bars->s_full[b], use, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
       uint32_t s[4][32];
@@ -306,66 +437,87 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       for (int c = 0; c < 4; ++c) tmem_ld_32x32(t_lane + b * kKTile + c * 32, s[c]);
       tmem_ld_wait();
 
-      // number of visible keys of this tile for this row (none for the unused rows of the tile, whose scores
-      // come from whatever the Q box left there)
-      const int lim = !row_ok ? 0 : (t < ctx_tiles) ? ctx - t * kKTile : pos + 1 - (t - ctx_tiles) * kKTile;
-      if (lim < kKTile) {
+      // Number of visible keys of this tile for this row. The branch is taken by whole warps: the code after it
+      // contains warp-wide tensor-memory stores.
+      const int lim = (t < ctx_tiles) ? ctx - t * kKTile : pos + 1 - (t - ctx_tiles) * kKTile;
+      if (__any_sync(0xffffffffu, lim < kKTile)) {
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
           for (int e = 0; e < 32; ++e)
             if (c * 32 + e >= lim) s[c][e] = 0xff800000u;
       }
-      float mx4[4];
+      // A row that has not seen a visible key yet takes the maximum of this tile as its reference.
+      if (__any_sync(0xffffffffu, m_ref == -INFINITY)) {
+        float mx4[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float a = fmaxf(__uint_as_float(s[c][0]), __uint_as_float(s[c][1]));
+        for (int c = 0; c < 4; ++c) {
+          float a = fmaxf(__uint_as_float(s[c][0]), __uint_as_float(s[c][1]));
 #pragma unroll
-        for (int e = 2; e < 32; e += 2)
-          a = fmaxf(a, fmaxf(__uint_as_float(s[c][e]), __uint_as_float(s[c][e + 1])));
-        mx4[c] = a;
+          for (int e = 2; e < 32; e += 2)
+            a = fmaxf(a, fmaxf(__uint_as_float(s[c][e]), __uint_as_float(s[c][e + 1])));
+          mx4[c] = a;
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        if (m_ref == -INFINITY && row_ok) m_ref = mx;      // may stay -inf (no visible key in this tile either)
       }
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      // Move the reference only when the maximum has outgrown it by the threshold (or on first sight).
-      const bool grow = (mx > -INFINITY) && (m_ref == -INFINITY || (mx - m_ref) * sc > kRescaleThreshold);
-      if (__any_sync(0xffffffffu, grow && j > 0)) {
-        // O holds tiles < j scaled to the old reference: wait for P V of tile j-1, then rescale in place.
-        const int ib = (j - 1) & 1;
-        const uint32_t iuse = static_cast<uint32_t>((j - 1) >> 1) & 1u;
-        if (!mbar_wait(&bars->pv_done[ib], iuse, abort_flag, p.status)) { ok = false; break; }
-        tc_fence_after();
-        const float alpha = (grow && m_ref != -INFINITY) ? fast_exp2((m_ref - mx) * sc) : 1.0f;
+      // One pass: exponentials against the standing reference, their sum, and the largest exponent met. P_j replaces
+      // S_j in tensor memory: keys 2e, 2e+1 of this row share one 32-bit column.
+      float ref = (m_ref == -INFINITY) ? 0.f : m_ref * sc;
+      float xmax, tile_sum;
+      auto exp_pass = [&]() {
+        float xm4[4], sum4[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
+          float sa = 0.f, sb = 0.f, xa = -INFINITY, xb = -INFINITY;
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float x0 = fmaf(__uint_as_float(s[c][2 * e]), sc, -ref);
+            const float x1 = fmaf(__uint_as_float(s[c][2 * e + 1]), sc, -ref);
+            xa = fmaxf(xa, x0);
+            xb = fmaxf(xb, x1);
+            const float a0 = fast_exp2(x0), a1 = fast_exp2(x1);
+            sa += a0;
+            sb += a1;
+            pk[e] = pack_f16x2(a0, a1);
+          }
+          sum4[c] = sa + sb;
+          xm4[c] = fmaxf(xa, xb);
+          tmem_st_32x16(t_lane + b * kKTile + c * 16, pk);
+        }
+        xmax = fmaxf(fmaxf(xm4[0], xm4[1]), fmaxf(xm4[2], xm4[3]));
+        tile_sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      };
+      exp_pass();
+      // The reference only moves when some exponent outgrew it by more than the threshold: then O (which holds the
+      // tiles before this one, scaled to the old reference) and the running sum are rescaled, and P_j is redone.
+      const bool grow = row_ok && xmax > kRescaleThreshold;
+      if (__any_sync(0xffffffffu, grow)) {
+        if (j > 0) {
+          const int ib = (j - 1) % kSBufs;
+          const uint32_t iuse = static_cast<uint32_t>((j - 1) / kSBufs) & 1u;
+          if (!mbar_wait(&bars->pv_done[ib], iuse, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const float alpha = grow ? fast_exp2(-xmax) : 1.0f;
 #pragma unroll 1
-        for (int c = 0; c < HD / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld_32x32(t_lane + L::kOCol + c * 32, o);
-          tmem_ld_wait();
+          for (int c = 0; c < HD / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld_32x32(t_lane + L::kOCol + c * 32, o);
+            tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st_32x32(t_lane + L::kOCol + c * 32, o);
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st_32x32(t_lane + L::kOCol + c * 32, o);
+          }
+          l *= alpha;
         }
-        l *= alpha;
-      }
-      if (grow) m_ref = mx;
-      const float ref = (m_ref == -INFINITY) ? 0.f : m_ref * sc;
-      float sum4[4];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
-        float sa = 0.f, sb = 0.f;
-#pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const float a0 = fast_exp2(fmaf(__uint_as_float(s[c][2 * e]), sc, -ref));
-          const float a1 = fast_exp2(fmaf(__uint_as_float(s[c][2 * e + 1]), sc, -ref));
-          sa += a0;
-          sb += a1;
-          pk[e] = pack_f16x2(a0, a1);
+        if (grow) {
+          ref += xmax;
+          m_ref = ref / sc;
         }
-        sum4[c] = sa + sb;
-        // P_j replaces S_j: keys 2e, 2e+1 of this row share one 32-bit column.
-        tmem_st_32x16(t_lane + b * kKTile + c * 16, pk);
+        exp_pass();
       }
-      l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      l += tile_sum;
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
@@ -374,8 +526,8 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
 
     // ---- epilogue: O is final once P V of the last tile has completed
     if (ok) {
-      const int ib = (n_tiles - 1) & 1;
-      const uint32_t iuse = static_cast<uint32_t>((n_tiles - 1) >> 1) & 1u;
+      const int ib = (n_tiles - 1) % kSBufs;
+      const uint32_t iuse = static_cast<uint32_t>((n_tiles - 1) / kSBufs) & 1u;
       ok = mbar_wait(&bars->pv_done[ib], iuse, abort_flag, p.status);
     }
     const int q_dim = p.n_q_heads * HD;

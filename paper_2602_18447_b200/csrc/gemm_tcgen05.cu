@@ -53,6 +53,33 @@ __device__ __forceinline__ void st_v4(void* p, uint32_t a, uint32_t b, uint32_t 
 }
 __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
 
+// One 64-deep block of products D (+)= A B^T (four K = 16 steps; the descriptors advance by 32 bytes per step),
+// then an arrival on `commit_bar` once they have completed. Before them a non-blocking test of `peek_bar` is
+// issued; its answer (1 = that phase is complete) is only read after everything else has been issued.
+__device__ __forceinline__ bool umma_kblock_peek(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate_first, uint64_t* commit_bar, uint64_t* peek_bar,
+                                                 uint32_t peek_parity) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred P, Q;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "setp.ne.b32 Q, %7, 0;\n\t"
+      "add.u64 a1, %4, 2;\n\tadd.u64 b1, %5, 2;\n\t"
+      "add.u64 a2, %4, 4;\n\tadd.u64 b2, %5, 4;\n\t"
+      "add.u64 a3, %4, 6;\n\tadd.u64 b3, %5, 6;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, Q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], a1, b1, %6, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], a2, b2, %6, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], a3, b3, %6, 1;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ready)
+      : "r"(smem_u32(peek_bar)), "r"(peek_parity), "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc),
+        "r"(accumulate_first), "r"(smem_u32(commit_bar))
+      : "memory");
+  return ready != 0;
+}
+
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -105,6 +132,8 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
+    // One thread issues the two or three 16 KB boxes of a stage in turn. (Spreading them over lanes of the warp,
+    // which pays for 4 KB boxes, was measured slower here.)
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
@@ -119,14 +148,9 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           uint8_t* sb = sa + kABytes;
           mbar_arrive_expect_tx(&full_bar[stage], L::kStageBytes);
           tma_load_2d(sa, &tm_a, &full_bar[stage], kb * BK, m0);
-          if (EPI == kEpiSwiGLU) {
-            tma_load_2d(sb, &tm_b, &full_bar[stage], kb * BK, n0);
-            tma_load_2d(sb + 128 * BK * 2, &tm_b2, &full_bar[stage], kb * BK, n0);
-          } else {
-#pragma unroll
-            for (int h = 0; h < BN / 128; ++h)
-              tma_load_2d(sb + h * 128 * BK * 2, &tm_b, &full_bar[stage], kb * BK, n0 + h * 128);
-          }
+          tma_load_2d(sb, &tm_b, &full_bar[stage], kb * BK, n0);
+          if (EPI == kEpiSwiGLU) tma_load_2d(sb + 128 * BK * 2, &tm_b2, &full_bar[stage], kb * BK, n0);
+          else if (BN == 256) tma_load_2d(sb + 128 * BK * 2, &tm_b, &full_bar[stage], kb * BK, n0 + 128);
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
         u += sg.len;
@@ -138,28 +162,32 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
+    // The thread that feeds the tensor core must not stall: a wait on a barrier that is already complete still
+    // costs a round trip of a few hundred cycles, in which the short queue of issued products runs dry. So the
+    // test of the NEXT stage's barrier is issued before this stage's products and its answer is read after them.
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
+      const uint32_t smem_base = smem_u32(smem);
+      const uint64_t adesc0 = umma_desc_k128(smem_base);
+      const uint64_t bdesc0 = umma_desc_k128(smem_base + kABytes);
+      bool ready = false;
       for (int u = start; u < end && ok;) {
         const Segment sg = next_segment(u, end, kblocks);
         if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int i = 0; i < sg.len; ++i) {
-          if (!mbar_wait(&full_bar[stage], phase, abort_flag, status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
-          const uint64_t adesc = umma_desc_k128(sa);
-          const uint64_t bdesc = umma_desc_k128(sa + kABytes);
-#pragma unroll
-          for (int k = 0; k < BK / 16; ++k)
-            umma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (i | k) != 0);
-          umma_commit(&empty_bar[stage]);
-          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+          if (!ready && !mbar_wait(&full_bar[stage], phase, abort_flag, status)) { ok = false; break; }
+          const int ns = (stage + 1 == L::kStages) ? 0 : stage + 1;
+          const uint32_t np = (ns == 0) ? phase ^ 1u : phase;
+          const uint64_t off = static_cast<uint64_t>(stage * (L::kStageBytes >> 4));
+          ready = umma_kblock_peek(d_tmem, adesc0 + off, bdesc0 + off, kIdesc, i != 0, &empty_bar[stage], &full_bar[ns], np);
+          stage = ns;
+          phase = np;
         }
         if (!ok) break;
         umma_commit(&acc_full[acc]);

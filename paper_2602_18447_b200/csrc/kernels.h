@@ -23,14 +23,16 @@ struct AttnItem {
   int32_t slot;       // this piece's partial-result slot (unused when n_splits == 1)
   int32_t slot0;      // first slot of the query tile
   int32_t n_splits;   // pieces the query tile's key range is cut into (1 = whole range, at most 32)
+  int32_t tok0;       // first row of the step in the batch's token order
+  int32_t n_new;      // new tokens of the step
+  int32_t ctx;        // cached context length of the step's sequence
+  int32_t seq;        // row of the page table
+  int32_t pad[4];
 };
 
 struct AttnParams {
   const uint16_t* qkv;      // [T, n_qkv] fp16: q heads, k heads, v heads (q, k already rotated)
   uint16_t* out;            // [T, Hq*hd] fp16
-  const int32_t* cu_new;    // [B+1]
-  const int32_t* ctx_len;   // [B]
-  const int32_t* seq_id;    // [B]
   const int32_t* page_table;// [max_seqs, max_pages_per_seq]
   int32_t max_pages_per_seq;
   int32_t n_q_heads, n_kv_heads, head_dim, n_qkv;
