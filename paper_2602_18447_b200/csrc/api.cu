@@ -158,10 +158,14 @@ struct BatchLayout {
 };
 
 // Cost of an attention work item in key tiles: the tiles themselves plus the fixed part of a CTA (set-up, Q load,
-// pipeline fill, epilogue), and what the last piece of a split query tile adds by combining the partial results.
-constexpr double kAttnItemFixed = 3.0;
+// pipeline fill, epilogue), what being a piece of a split query tile adds (the partial result goes through global
+// memory), and what the last piece adds by combining the partial results.
+// Measured on B200: a tile takes ~2 k cycles; set-up to first S ~5.5 k; the epilogue of a piece (partial store,
+// fence, counter) ~7 k against ~1.5 k for a whole range.
+constexpr double kAttnItemFixed = 3.5;
+constexpr double kAttnPieceExtra = 3.0;
 constexpr double kAttnMergeFixed = 1.0;
-constexpr double kAttnMergePerSplit = 0.4;
+constexpr double kAttnMergePerSplit = 0.5;
 
 // Time at which the last SM finishes when the items, sorted by decreasing cost, are handed to whichever of
 // `machines` SMs is free first (what the hardware does with one CTA per SM and the grid in that order).
@@ -209,6 +213,7 @@ void build_attention_work(const cs_model* m, int B, const int32_t* lens, const i
       for (int s = 0; s < n; ++s) {
         const int len = static_cast<int>(static_cast<long>(u.nt) * (s + 1) / n - static_cast<long>(u.nt) * s / n);
         double c = kAttnItemFixed + len;
+        if (n > 1) c += kAttnPieceExtra;
         if (n > 1 && s == n - 1) c += kAttnMergeFixed + kAttnMergePerSplit * n;
         for (int h = 0; h < heads; ++h) cost.push_back(c);
       }
