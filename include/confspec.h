@@ -201,6 +201,19 @@ int cs_last_status(cs_model* model, void* stream);
  * K and N multiples of 8. Asynchronous on `stream`. */
 int cs_gemm_f16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* out,
                  int M, int N, int K, int epilogue, void* stream);
+/* The last stage of the pass on its own (Section 4.2, Eqs. 2-4): logits z = w_lm h for B steps, logsumexp over the
+ * whole vocabulary fused into the product (the logits are never written), conf = max_j exp(z[verdict_ids[j]] - lse),
+ * verdict = first j attaining it, accept = (conf >= tau).
+ *   w_lm               device fp16 [vocab, d_model], row-major.
+ *   h                  device fp16 [B, d_model]: the final-normed hidden state of each step's last position.
+ *   verdict_ids        host int32[n_verdict], 1 <= n_verdict <= 8.
+ *   out_conf, out_accept, out_verdict (or NULL), out_lse (or NULL)   device arrays of B entries.
+ * d_model a multiple of 8. The per-CTA partial sums live in a scratch buffer that the library allocates on first use
+ * (cudaMalloc) and keeps; calls on different streams that overlap on the GPU would share it and race.
+ * Asynchronous on `stream`. */
+int cs_lm_head_gate(const uint16_t* w_lm, const uint16_t* h, int B, int d_model, int vocab, const int32_t* verdict_ids,
+                    int n_verdict, float tau, float* out_conf, uint8_t* out_accept, int32_t* out_verdict, float* out_lse,
+                    void* stream);
 /* out fp16 [rows, d] = RMSNorm(x fp32 [rows, d]; gain fp32 [d], eps). */
 int cs_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps, void* stream);
 /*

@@ -870,6 +870,51 @@ int cs_gemm_f16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* 
   return CS_OK;
 }
 
+int cs_lm_head_gate(const uint16_t* w_lm, const uint16_t* h, int B, int d_model, int vocab, const int32_t* verdict_ids,
+                    int n_verdict, float tau, float* out_conf, uint8_t* out_accept, int32_t* out_verdict, float* out_lse,
+                    void* stream) {
+  if (!w_lm || !h || B < 0 || d_model < 8 || (d_model % 8) || vocab < 1 || tau != tau) return CS_EINVAL;
+  if (n_verdict < 1 || n_verdict > 8 || !verdict_ids) return CS_EINVAL;
+  for (int j = 0; j < n_verdict; ++j)
+    if (verdict_ids[j] < 0 || verdict_ids[j] >= vocab) return CS_EINVAL;
+  if (B == 0) return CS_OK;
+  if (!out_conf || !out_accept) return CS_EINVAL;
+  if (!g_test_status) {
+    CS_CUDA(cudaMalloc(reinterpret_cast<void**>(&g_test_status), 256));
+    CS_CUDA(cudaMemset(g_test_status, 0, 256));
+  }
+  // scratch: per-CTA (max, sum exp) pairs and the verdict logits of one chunk of up to 64 steps
+  static DevBuf scratch;
+  const size_t part_floats = static_cast<size_t>(2) * kNumSMs * 64;
+  int rc;
+  if ((rc = scratch.ensure((part_floats + 64 * 8) * sizeof(float)))) return rc;
+  float* part_max = static_cast<float*>(scratch.p);
+  float* part_sum = part_max + kNumSMs * 64;
+  float* vlog = part_max + part_floats;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  CUtensorMap tm_w, tm_h;
+  if (!make_gemm_operand_map(&tm_w, w_lm, vocab, d_model)) {
+    g_cuda_error = "cuTensorMapEncodeTiled failed for the LM head";
+    return CS_ECUDA;
+  }
+  int tiles_per_cta;
+  const int grid = lm_head_grid(vocab, &tiles_per_cta);
+  for (int b0 = 0; b0 < B; b0 += 64) {
+    const int bc = std::min(64, B - b0);
+    const int bp = lm_head_batch_pad(bc);
+    // rows past B are filled with zeros by the copy engine
+    if (!make_tensor_map_16b(&tm_h, h, B, d_model, bp, 64, true, false)) {
+      g_cuda_error = "cuTensorMapEncodeTiled failed for the hidden states";
+      return CS_ECUDA;
+    }
+    CS_CUDA(launch_lm_head(tm_w, tm_h, b0, bc, bp, d_model, vocab, verdict_ids, n_verdict, part_max, part_sum, vlog,
+                           nullptr, g_test_status, s));
+    CS_CUDA(launch_gate(part_max, part_sum, grid, bp, vlog, n_verdict, bc, tau, out_conf + b0, out_accept + b0,
+                        out_verdict ? out_verdict + b0 : nullptr, out_lse ? out_lse + b0 : nullptr, s));
+  }
+  return CS_OK;
+}
+
 int cs_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps, void* stream) {
   if (!x || !gain || !out || rows < 0 || d < 4 || (d % 4)) return CS_EINVAL;
   CS_CUDA(launch_rmsnorm(x, gain, out, rows, d, eps, static_cast<cudaStream_t>(stream)));

@@ -1,0 +1,74 @@
+"""Parity at the full sizes of the 1.5B-shaped workloads (all 28 layers, the whole batch, the launch configuration
+the benchmark times): the CUDA path runs the complete batch, the CPU oracle recomputes a sample of its steps one by
+one (steps are independent), and the two are compared with the specified tolerances. The tau sweep of the batch-64
+workload goes through cs_escalate_mask on the stored confidences."""
+import numpy as np
+import pytest
+
+from workloads import get_config, make_batch, model_weights
+
+import parity_common as P
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def weights_1p5b():
+    cfg = get_config("cfg2_1p5b_b16")
+    return model_weights(cfg.model, cfg.seed)
+
+
+def _run_full(name, weights, sample):
+    cfg = get_config(name)
+    batch = make_batch(cfg)
+    ses = P.build_session(cfg, weights, batch)
+    try:
+        ses.verify()
+        gpu = ses.results()
+        logits, lse = ses.last_logits(), ses.last_lse()
+        ref = P.oracle_outputs(cfg, weights, batch, steps=sample)
+        stats = P.compare(gpu, logits, ref, cfg.tau, steps=sample, gpu_lse=lse)
+        P.check_verdict(gpu, ref, cfg.verdict_ids, steps=sample)
+        # properties that hold for every step of the batch, sampled or not
+        assert np.all(np.isfinite(gpu["conf"])) and np.all(gpu["conf"] > 0) and np.all(gpu["conf"] <= 1)
+        assert np.array_equal(gpu["accept"], (gpu["conf"] >= np.float32(cfg.tau)).astype(np.uint8))
+        z = logits.astype(np.float64)
+        lse_from_logits = np.log(np.exp(z - z.max(axis=1, keepdims=True)).sum(axis=1)) + z.max(axis=1)
+        assert np.max(np.abs(lse_from_logits - lse)) < 1e-4          # fused logsumexp == logsumexp of the logits
+        vid = list(cfg.verdict_ids)
+        assert np.max(np.abs(np.exp(z[:, vid] - lse_from_logits[:, None]).max(axis=1) - gpu["conf"])) < 1e-6
+        return cfg, ses, gpu, ref, stats
+    except BaseException:
+        ses.close()
+        raise
+
+
+def test_cfg2_batch16_full_depth(weights_1p5b):
+    cfg, ses, gpu, ref, stats = _run_full("cfg2_1p5b_b16", weights_1p5b, sample=[0, 7, 15])
+    ses.close()
+    assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
+
+
+def test_cfg3_batch64_full_depth_and_tau_sweep(weights_1p5b):
+    import torch
+    from paper_2602_18447_b200 import binding as B
+    cfg, ses, gpu, ref, stats = _run_full("cfg3_1p5b_b64", weights_1p5b, sample=[3, 40])
+    try:
+        n = cfg.batch
+        for tau in cfg.taus:
+            acc = torch.zeros(n, dtype=torch.uint8, device="cuda")
+            idx = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+            cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+            B.cs_escalate_mask(ses.out_conf, tau, acc, idx, cnt)
+            torch.cuda.synchronize()
+            want_acc, want_idx, want_cnt = P.O.escalate_list(gpu["conf"], tau)
+            assert int(cnt.item()) == want_cnt and np.array_equal(acc.cpu().numpy(), want_acc)
+            assert np.array_equal(idx.cpu().numpy()[:want_cnt], want_idx)
+    finally:
+        ses.close()
+
+
+def test_cfg4_long_context_full_depth(weights_1p5b):
+    cfg, ses, gpu, ref, stats = _run_full("cfg4_1p5b_long", weights_1p5b, sample=[1, 6])
+    ses.close()
+    assert stats["logit_err"] <= P.LOGIT_TOL

@@ -93,3 +93,41 @@ def test_escalate_mask_matches_oracle_bit_exact():
             assert np.array_equal(acc.cpu().numpy(), want_acc)
             assert np.array_equal(idx.cpu().numpy()[:want_cnt], want_idx)
             assert np.all(idx.cpu().numpy()[want_cnt:] == -1)
+
+
+@pytest.mark.parametrize("B,d,vocab", [(1, 256, 4096), (16, 1536, 151936), (33, 1536, 20488), (64, 3584, 30000),
+                                       (100, 256, 4100)])
+def test_lm_head_gate_matches_oracle(B, d, vocab):
+    """Logits of B hidden states against the whole vocabulary, fused logsumexp, confidence and gate. Two LM-head rows
+    are planted so that confidences land on both sides of the threshold; the vocabulary has a ragged last tile."""
+    import torch
+    from paper_2602_18447_b200 import binding as Bd
+    g = np.random.default_rng(B * 31 + d + vocab)
+    w = _f16_randn(g, (vocab, d), 0.02)
+    h = _f16_randn(g, (B, d), 1.0)
+    vids = [1, vocab - 1, 7]
+    u = g.standard_normal(d)
+    u /= np.linalg.norm(u)
+    beta = np.log(vocab) + 0.5
+    w[vids[0]] = (beta * u).astype(np.float16)      # h has unit-variance entries, so u.h ~ N(0, 1)
+    w[vids[1]] = (-beta * u).astype(np.float16)
+    z = h.astype(np.float64) @ w.astype(np.float64).T
+    conf, verdict, lse = O.verdict_confidence(z, vids)
+    out_conf = torch.empty(B, dtype=torch.float32, device="cuda")
+    out_acc = torch.empty(B, dtype=torch.uint8, device="cuda")
+    out_v = torch.empty(B, dtype=torch.int32, device="cuda")
+    out_lse = torch.empty(B, dtype=torch.float32, device="cuda")
+    for tau in (0.3, 0.9):
+        Bd.cs_lm_head_gate(_to_dev(w), _to_dev(h), vids, tau, out_conf, out_acc, out_v, out_lse)
+        torch.cuda.synchronize()
+        got = out_conf.cpu().numpy().astype(np.float64)
+        # fp32 accumulation of exact fp16 products, exponentials in fp32
+        assert np.max(np.abs(out_lse.cpu().numpy() - lse)) < 2e-4
+        assert np.max(np.abs(got - conf)) < 2e-4 * np.maximum(conf, 1e-3).max()
+        sure = np.abs(conf - tau) > 1e-3
+        assert np.array_equal(out_acc.cpu().numpy()[sure], O.gate(conf, tau)[sure])
+        pv = np.sort(np.exp(z[:, vids] - lse[:, None]), axis=1)
+        clear = (pv[:, -1] - pv[:, -2]) > 1e-4
+        assert np.array_equal(out_v.cpu().numpy()[clear], verdict[clear])
+    if B > 4:
+        assert 0 < (conf >= 0.3).sum() < B
