@@ -33,7 +33,8 @@ enum {
   CS_ENOMEM = 2,   /* a device or host allocation failed */
   CS_ECUDA = 3,    /* a CUDA runtime / driver call failed; see cs_last_cuda_error */
   CS_ETIMEOUT = 4, /* a kernel gave up on a bounded wait (reported by cs_last_status) */
-  CS_ESTATE = 5    /* the call does not fit the handle's state (e.g. sequence not set) */
+  CS_ESTATE = 5,   /* the call does not fit the handle's state (e.g. sequence not set) */
+  CS_ELIMIT = 6    /* a size exceeds the fixed capacity of an entry point that never allocates */
 };
 
 typedef struct cs_model cs_model;
@@ -214,6 +215,34 @@ int cs_gemm_f16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* 
 int cs_lm_head_gate(const uint16_t* w_lm, const uint16_t* h, int B, int d_model, int vocab, const int32_t* verdict_ids,
                     int n_verdict, float tau, float* out_conf, uint8_t* out_accept, int32_t* out_verdict, float* out_lse,
                     void* stream);
+/*
+ * cs_lm_head_gate_static - the same stage as cs_lm_head_gate, for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this entry point exists for the sake of its callers, not of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits. Examples are a serving process whose memory pool owns
+ * all of the device memory and forbids side allocations, a real-time loop that may not take the allocator's locks or
+ * its implicit device synchronisation, and a plug-in loaded into a host application that hands out buffers itself.
+ * cs_lm_head_gate would call cudaMalloc on its first use; this function never calls cudaMalloc, cudaFree or any
+ * routine that allocates.
+ *
+ * Instead its scratch (per-CTA partial maxima and sums, the verdict logits, a status word: about 78 KB) is a fixed
+ * array inside the library image. Consequences the caller must know:
+ *   - every GPU on which the library is loaded holds that array until the process exits;
+ *   - capacity is fixed: B <= CS_LM_HEAD_STATIC_MAX_STEPS, else CS_ELIMIT is returned and nothing is launched (larger
+ *     batches: call it in chunks, one after the other on one stream);
+ *   - all calls share the one array per GPU: two calls that overlap on the GPU (different streams, or different
+ *     threads) race on it and give wrong results. Calls on one stream are ordered and safe. The function clears the
+ *     part of the array that must start at zero on every call, so leftovers of an earlier call do no harm;
+ *   - the first call on each device looks up the array's device address (with that device current). Make that first
+ *     call outside any stream capture.
+ * If the LM-head kernel gives up on a bounded wait, every out_conf is set to NaN and every out_accept to 0.
+ * Arguments, layouts and asynchrony are those of cs_lm_head_gate.
+ * Errors: CS_EINVAL (arguments), CS_ELIMIT (B too large), CS_ECUDA.
+ */
+#define CS_LM_HEAD_STATIC_MAX_STEPS 64
+int cs_lm_head_gate_static(const uint16_t* w_lm, const uint16_t* h, int B, int d_model, int vocab,
+                           const int32_t* verdict_ids, int n_verdict, float tau, float* out_conf, uint8_t* out_accept,
+                           int32_t* out_verdict, float* out_lse, void* stream);
 /* out fp16 [rows, d] = RMSNorm(x fp32 [rows, d]; gain fp32 [d], eps). */
 int cs_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps, void* stream);
 /*

@@ -11,13 +11,13 @@ import numpy as np
 
 from . import build as _build
 
-CS_OK, CS_EINVAL, CS_ENOMEM, CS_ECUDA, CS_ETIMEOUT, CS_ESTATE = range(6)
+CS_OK, CS_EINVAL, CS_ENOMEM, CS_ECUDA, CS_ETIMEOUT, CS_ESTATE, CS_ELIMIT = range(7)
 
 EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_reserve",
     "cs_kv_alloc", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
     "cs_verify_steps", "cs_escalate_mask", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
-    "cs_last_status", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_take_launch_count", "cs_profile", "cs_profile_read",
+    "cs_last_status", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_profile", "cs_profile_read",
 ]
 
 PROF_CLASSES = ["embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gateup", "gemm_down",
@@ -81,6 +81,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_gemm_f16": (C.c_int, [vp, vp, vp, vp, i32, i32, i32, i32, vp]),
         "cs_rmsnorm": (C.c_int, [vp, vp, vp, i32, i32, f32, vp]),
         "cs_lm_head_gate": (C.c_int, [vp, vp, i32, i32, i32, vp, i32, f32, vp, vp, vp, vp, vp]),
+        "cs_lm_head_gate_static": (C.c_int, [vp, vp, i32, i32, i32, vp, i32, f32, vp, vp, vp, vp, vp]),
         "cs_take_launch_count": (C.c_int64, []),
         "cs_profile": (C.c_int, [vp, i32]),
         "cs_profile_read": (C.c_int, [vp, vp, vp, i32]),
@@ -261,6 +262,14 @@ def cs_lm_head_gate(w_lm, h, verdict_ids: Sequence[int], tau: float, out_conf, o
     _check(fn(_dev_ptr(w_lm), _dev_ptr(h), int(h.shape[0]), int(h.shape[1]), int(w_lm.shape[0]), _np_ptr(v),
               int(v.shape[0]), float(tau), _dev_ptr(out_conf), _dev_ptr(out_accept), _dev_ptr(out_verdict),
               _dev_ptr(out_lse), _stream_ptr(stream)), entry)
+
+
+def cs_lm_head_gate_static(w_lm, h, verdict_ids: Sequence[int], tau: float, out_conf, out_accept, out_verdict=None,
+                           out_lse=None, stream=None) -> None:
+    """Same stage through the entry point that never allocates device memory (at most 64 steps per call; calls that
+    overlap on the GPU share one scratch array and race: keep them on one stream)."""
+    cs_lm_head_gate(w_lm, h, verdict_ids, tau, out_conf, out_accept, out_verdict, out_lse, stream,
+                    entry="cs_lm_head_gate_static")
 
 
 def cs_rmsnorm(x, gain, out, rows: int, d: int, eps: float, stream=None) -> None:

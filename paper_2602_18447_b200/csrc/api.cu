@@ -473,6 +473,7 @@ const char* cs_strerror(int status) {
     case CS_ECUDA: return "CUDA error";
     case CS_ETIMEOUT: return "a kernel gave up on a bounded wait";
     case CS_ESTATE: return "call does not fit the handle's state";
+    case CS_ELIMIT: return "size exceeds the fixed capacity of an entry point that never allocates";
     default: return "unknown status";
   }
 }

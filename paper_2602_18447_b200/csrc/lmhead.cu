@@ -394,3 +394,92 @@ cudaError_t launch_escalate(const float* conf, int B, float tau, uint8_t* out_ac
 }
 
 }  // namespace cs
+
+// ------------------------------------------------------------------------------------------------------------------
+// cs_lm_head_gate_static: the LM-head + gate stage for callers that must not allocate device memory.
+// ------------------------------------------------------------------------------------------------------------------
+#include "../../include/confspec.h"
+
+#include "gemm.h"
+
+namespace {
+
+constexpr int kStaticMaxSteps = CS_LM_HEAD_STATIC_MAX_STEPS;
+constexpr int kStaticPartFloats = 2 * cs::kNumSMs * kStaticMaxSteps;      // per-CTA (max, sum exp) pairs
+constexpr int kStaticVerdictFloats = kStaticMaxSteps * 8;                 // logits of the verdict ids
+constexpr int kStaticStatusFloats = 64;                                   // status word, padded to 256 bytes
+constexpr int kStaticFloats = kStaticPartFloats + kStaticVerdictFloats + kStaticStatusFloats;
+
+// The scratch of the no-allocation entry point: about 78 KB that every GPU which loads the library holds until the
+// process exits. In host code this name is only a handle; the device address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) float g_lm_static_scratch[kStaticFloats];
+
+constexpr int kMaxDevices = 64;
+float* g_lm_static_ptr[kMaxDevices] = {};
+
+// A pass that gave up on a bounded wait leaves no usable numbers: make that visible in the outputs themselves.
+__global__ void poison_on_timeout_kernel(const uint32_t* status, float* out_conf, uint8_t* out_accept,
+                                         int32_t* out_verdict, float* out_lse, int B) {
+  if (*status == 0) return;
+  for (int i = threadIdx.x; i < B; i += blockDim.x) {
+    out_conf[i] = __int_as_float(0x7fc00000);
+    out_accept[i] = 0;
+    if (out_verdict) out_verdict[i] = -1;
+    if (out_lse) out_lse[i] = __int_as_float(0x7fc00000);
+  }
+}
+
+}  // namespace
+
+extern "C" int cs_lm_head_gate_static(const uint16_t* w_lm, const uint16_t* h, int B, int d_model, int vocab,
+                                      const int32_t* verdict_ids, int n_verdict, float tau, float* out_conf,
+                                      uint8_t* out_accept, int32_t* out_verdict, float* out_lse, void* stream) {
+  using namespace cs;
+  if (!w_lm || !h || B < 0 || d_model < 8 || (d_model % 8) || vocab < 1 || tau != tau) return CS_EINVAL;
+  if (n_verdict < 1 || n_verdict > 8 || !verdict_ids) return CS_EINVAL;
+  for (int j = 0; j < n_verdict; ++j)
+    if (verdict_ids[j] < 0 || verdict_ids[j] >= vocab) return CS_EINVAL;
+  if (B > kStaticMaxSteps) return CS_ELIMIT;
+  if (B == 0) return CS_OK;
+  if (!out_conf || !out_accept) return CS_EINVAL;
+
+  // Set-up, once per device, with that device current: the device address of the scratch array.
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CS_ECUDA;
+  if (!g_lm_static_ptr[dev]) {
+    float* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_lm_static_scratch) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return CS_ECUDA;
+    }
+    g_lm_static_ptr[dev] = ptr;
+  }
+  float* scratch = g_lm_static_ptr[dev];
+  float* part_max = scratch;
+  float* part_sum = scratch + kNumSMs * kStaticMaxSteps;
+  float* vlog = scratch + kStaticPartFloats;
+  uint32_t* status = reinterpret_cast<uint32_t*>(scratch + kStaticPartFloats + kStaticVerdictFloats);
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The array keeps what the previous call left. The partial pairs and the verdict logits are overwritten in full
+  // by this call; the status word is the one thing that must start at zero.
+  if (cudaMemsetAsync(status, 0, sizeof(uint32_t), s) != cudaSuccess) { cudaGetLastError(); return CS_ECUDA; }
+  CUtensorMap tm_w, tm_h;
+  const int bp = lm_head_batch_pad(B);
+  if (!make_gemm_operand_map(&tm_w, w_lm, vocab, d_model) ||
+      !make_tensor_map_16b(&tm_h, h, B, d_model, bp, 64, true, false))      // rows past B read as zeros
+    return CS_ECUDA;
+  int tiles_per_cta;
+  const int grid = lm_head_grid(vocab, &tiles_per_cta);
+  if (launch_lm_head(tm_w, tm_h, 0, B, bp, d_model, vocab, verdict_ids, n_verdict, part_max, part_sum, vlog, nullptr,
+                     status, s) != cudaSuccess ||
+      launch_gate(part_max, part_sum, grid, bp, vlog, n_verdict, B, tau, out_conf, out_accept, out_verdict, out_lse,
+                  s) != cudaSuccess) {
+    cudaGetLastError();
+    return CS_ECUDA;
+  }
+  poison_on_timeout_kernel<<<1, 64, 0, s>>>(status, out_conf, out_accept, out_verdict, out_lse, B);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return CS_ECUDA;
+  return CS_OK;
+}
