@@ -45,13 +45,26 @@ __device__ __forceinline__ Segment next_segment(int u, int end, int kblocks) {
   return s;
 }
 
+// Order of the tiles. A CTA of the whole-tile epilogues (fp16 store, SwiGLU) takes consecutive tiles: with the column
+// tile running fastest it keeps its rows of A and walks through the weights, and the CTAs that hold other rows walk
+// through the same weights at the same time, so the weights stream from DRAM evenly over the whole launch (with the
+// row tile fastest, every CTA wanted its share of the weights in its first tile and waited for DRAM there).
+__device__ __forceinline__ int tile_m(int tile, int m_tiles, int n_tiles, int epi) {
+  return epi == kEpiResidAdd ? tile % m_tiles : tile / n_tiles;
+}
+__device__ __forceinline__ int tile_n(int tile, int m_tiles, int n_tiles, int epi) {
+  return epi == kEpiResidAdd ? tile / m_tiles : tile % n_tiles;
+}
+
 __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 __device__ __forceinline__ void st_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
-__device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
+// z * sigmoid(z) with the fast exponential and the fast reciprocal: an IEEE division here made the epilogue of a
+// SwiGLU tile as long as its main loop.
+__device__ __forceinline__ float silu_f(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
 // One 64-deep block of products D (+)= A B^T (four K = 16 steps; the descriptors advance by 32 bytes per step),
 // then an arrival on `commit_bar` once they have completed. Before them a non-blocking test of `peek_bar` is
@@ -84,7 +97,7 @@ template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                  const __grid_constant__ CUtensorMap tm_b2, void* __restrict__ out, int M, int N, int m_tiles,
-                 int kblocks, int total_units, int units_per_cta, uint32_t* status) {
+                 int n_tiles, int kblocks, int total_units, int units_per_cta, uint32_t* status) {
   using L = GemmSmem<BN>;
   constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
   constexpr uint32_t kTmemCols = 2 * BN;
@@ -140,8 +153,8 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       bool ok = true;
       for (int u = start; u < end && ok;) {
         const Segment sg = next_segment(u, end, kblocks);
-        const int m0 = (sg.tile % m_tiles) * BM;
-        const int n0 = (sg.tile / m_tiles) * OUT_BN;
+        const int m0 = tile_m(sg.tile, m_tiles, n_tiles, EPI) * BM;
+        const int n0 = tile_n(sg.tile, m_tiles, n_tiles, EPI) * OUT_BN;
         for (int kb = sg.kb0; kb < sg.kb0 + sg.len; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
           uint8_t* sa = smem + stage * L::kStageBytes;
@@ -204,8 +217,8 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     bool ok = true;
     for (int u = start; u < end && ok;) {
       const Segment sg = next_segment(u, end, kblocks);
-      const int m0 = (sg.tile % m_tiles) * BM;
-      const int n0 = (sg.tile / m_tiles) * OUT_BN;
+      const int m0 = tile_m(sg.tile, m_tiles, n_tiles, EPI) * BM;
+      const int n0 = tile_n(sg.tile, m_tiles, n_tiles, EPI) * OUT_BN;
       if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, status)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
@@ -326,7 +339,7 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
     grid = (tiles + tpc - 1) / tpc;
     upc = tpc * kblocks;
   }
-  gemm_f16_kernel<BN, EPI><<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tb, tb2, out, M, N, m_tiles, kblocks, total,
+  gemm_f16_kernel<BN, EPI><<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tb, tb2, out, M, N, m_tiles, n_tiles, kblocks, total,
                                                                       upc, status);
   count_launch();
   return cudaGetLastError();
