@@ -7,8 +7,8 @@
 // Work is measured in k-blocks (128 x BN x 64 products). Each CTA owns a contiguous range of k-blocks in the
 // order (n tile, m tile, k); a range may start or end inside a tile. For the two epilogues that need the whole
 // sum (fp16 store, SwiGLU) the ranges are whole tiles. For the residual epilogue (x += a * w^T, fp32) the
-// range is cut evenly over the SMs whatever the tile boundaries are, and every piece is added into x with
-// vector atomics, which is what lets the narrow O and down projections fill all SMs.
+// range is cut evenly over the SMs whatever the tile boundaries are, and every piece is added into x by the copy
+// engine (TMA reduce-add from a shared-memory box), which is what lets the narrow O and down projections fill all SMs.
 #include "gemm.h"
 
 #include "kernels.h"
@@ -30,7 +30,11 @@ struct GemmSmem {
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kStages = (BN == 256) ? 4 : 6;
   static constexpr int kBarBytes = 256;
-  static constexpr int kTotal = kStages * kStageBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
+  // Residual epilogue only: per epilogue warp two 32-row x 32-column fp32 boxes (4 KB each) from which the copy
+  // engine adds into the output.
+  static constexpr int kStagingBytes = 4 * 2 * 4096;
+  static constexpr int kStagingOff = kStages * kStageBytes;
+  static constexpr int kTotal = kStages * kStageBytes + kStagingBytes + kBarBytes + 1024;  // + slack for alignment
 };
 
 struct Segment {
@@ -56,8 +60,22 @@ __device__ __forceinline__ int tile_n(int tile, int m_tiles, int n_tiles, int ep
   return epi == kEpiResidAdd ? tile / m_tiles : tile % n_tiles;
 }
 
-__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+// out[tile] += shared-memory box, by the copy engine (element-wise fp32 atomics at L2, whole sectors at a time). The
+// box is [32 rows][32 floats] with the 128-byte swizzle; rows and columns past the tensor's extent are dropped.
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* m, const void* smem_src, int x, int y) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Until at most `N` of this thread's groups still have to read their shared-memory source.
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(p)), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ void st_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
@@ -96,8 +114,8 @@ __device__ __forceinline__ bool umma_kblock_peek(uint32_t tmem_d, uint64_t adesc
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                 const __grid_constant__ CUtensorMap tm_b2, void* __restrict__ out, int M, int N, int m_tiles,
-                 int n_tiles, int kblocks, int total_units, int units_per_cta, uint32_t* status) {
+                 const __grid_constant__ CUtensorMap tm_b2, const __grid_constant__ CUtensorMap tm_out,
+                 void* __restrict__ out, int M, int N, int m_tiles, int n_tiles, int kblocks, int total_units, int units_per_cta, uint32_t* status) {
   using L = GemmSmem<BN>;
   constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
   constexpr uint32_t kTmemCols = 2 * BN;
@@ -105,7 +123,7 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kStages * L::kStageBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kStagingOff + L::kStagingBytes);
   uint64_t* full_bar = bars;                       // [kStages] TMA -> MMA
   uint64_t* empty_bar = bars + L::kStages;         // [kStages] MMA -> TMA
   uint64_t* acc_full = bars + 2 * L::kStages;      // [2] MMA -> epilogue
@@ -265,20 +283,32 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           }
         }
       } else {
-        float* o = reinterpret_cast<float*>(out) + static_cast<size_t>(row) * N;
+        // x += acc. Each warp stages its 32 rows, 32 columns at a time, in shared memory and lets the copy engine add
+        // the box into x: per-lane atomics on 16-byte pieces of 32 different rows took as long as a third of the
+        // main loop. Two boxes per warp alternate; lane 0 owns the warp's copy groups.
+        uint8_t* stage0 = smem + L::kStagingOff + quad * 2 * 4096;
+        const int y = m0 + quad * 32;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = 0; c < BN / 32 && n0 + c * 32 < N; ++c) {
           tmem_ld_32x32(t_row + c * 32, r);
+          if (c >= 2) {
+            if (lane == 0) bulk_wait_group_read<1>();      // the box written two rounds ago has been read
+            __syncwarp();
+          }
           tmem_ld_wait();
-          const int col = n0 + c * 32;
-          if (row_ok) {
+          uint8_t* box = stage0 + (c & 1) * 4096;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-              if (col + j * 4 < N)
-                red_add_v4(o + col + j * 4, __uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                           __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(box + lane * 128 + ((j ^ (lane & 7)) << 4), r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {     // one group per round, empty or not: the wait above counts groups
+            if (y < M) tma_reduce_add_2d(&tm_out, box, n0 + c * 32, y);
+            bulk_commit_group();
           }
         }
+        if (lane == 0) bulk_wait_group_read<0>();
+        __syncwarp();
       }
       tc_fence_before();
       __syncwarp();
@@ -287,6 +317,7 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if (acc == 0) acc_phase ^= 1u;
       u += sg.len;
     }
+    if (EPI == kEpiResidAdd && lane == 0) bulk_wait_group_all();   // the additions have been performed
   }
 
   tc_fence_before();
@@ -311,6 +342,18 @@ EncodeTiledFn encode_fn() {
     return reinterpret_cast<EncodeTiledFn>(p);
   }();
   return fn;
+}
+
+// fp32 [rows, cols] row-major, boxes of 32 rows x 32 columns (128 bytes per row), 128-byte swizzle.
+bool make_out_f32_map(CUtensorMap* tm, void* base, int rows, int cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 4};
+  cuuint32_t box[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int BN, int EPI>
@@ -339,7 +382,9 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
     grid = (tiles + tpc - 1) / tpc;
     upc = tpc * kblocks;
   }
-  gemm_f16_kernel<BN, EPI><<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tb, tb2, out, M, N, m_tiles, n_tiles, kblocks, total,
+  CUtensorMap tout = ta;   // only the residual epilogue reads it
+  if (EPI == kEpiResidAdd && !make_out_f32_map(&tout, out, M, N)) return cudaErrorInvalidValue;
+  gemm_f16_kernel<BN, EPI><<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tb, tb2, tout, out, M, N, m_tiles, n_tiles, kblocks, total,
                                                                       upc, status);
   count_launch();
   return cudaGetLastError();
