@@ -24,23 +24,50 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const uint16_t*
   }
 }
 
-// One warp per row: sum of squares, then scale and round to bf16. The second pass re-reads the row from L2.
+// One warp per row. Rows of up to 4096 values are held in registers between the sum of squares and the scaling, so
+// x is read once and all of a row's loads are in flight together; longer rows are read twice.
+constexpr int kNormRegVecs = 32;   // float4 per lane
+
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
                                uint16_t* __restrict__ out, int rows, int d, float eps) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
   const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(row) * d);
+  const float4* g4 = reinterpret_cast<const float4*>(gain);
+  uint2* o = reinterpret_cast<uint2*>(out + static_cast<size_t>(row) * d);
+  const int n = d >> 2;
+  if (n <= 32 * kNormRegVecs) {
+    float4 v[kNormRegVecs];
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < kNormRegVecs; ++i) {
+      const int idx = lane + 32 * i;
+      if (idx < n) v[i] = xr[idx];
+    }
+#pragma unroll
+    for (int i = 0; i < kNormRegVecs; ++i)
+      if (lane + 32 * i < n) ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    ss = warp_sum(ss);
+    const float r = rsqrtf(ss / static_cast<float>(d) + eps);
+#pragma unroll
+    for (int i = 0; i < kNormRegVecs; ++i) {
+      const int idx = lane + 32 * i;
+      if (idx < n) {
+        const float4 g = g4[idx];
+        o[idx] = make_uint2(pack_f16x2(v[i].x * r * g.x, v[i].y * r * g.y), pack_f16x2(v[i].z * r * g.z, v[i].w * r * g.w));
+      }
+    }
+    return;
+  }
   float ss = 0.f;
-  for (int i = lane; i < d / 4; i += 32) {
+  for (int i = lane; i < n; i += 32) {
     const float4 v = xr[i];
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = warp_sum(ss);
   const float r = rsqrtf(ss / static_cast<float>(d) + eps);
-  const float4* g4 = reinterpret_cast<const float4*>(gain);
-  uint2* o = reinterpret_cast<uint2*>(out + static_cast<size_t>(row) * d);
-  for (int i = lane; i < d / 4; i += 32) {
+  for (int i = lane; i < n; i += 32) {
     const float4 v = xr[i];
     const float4 g = g4[i];
     o[i] = make_uint2(pack_f16x2(v.x * r * g.x, v.y * r * g.y), pack_f16x2(v.z * r * g.z, v.w * r * g.w));
@@ -144,7 +171,7 @@ cudaError_t launch_embed(const int32_t* tokens, const uint16_t* embed, float* x,
 cudaError_t launch_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps,
                            cudaStream_t s) {
   if (rows <= 0) return cudaSuccess;
-  const int warps = 8;
+  const int warps = 4;
   rmsnorm_kernel<<<(rows + warps - 1) / warps, warps * 32, 0, s>>>(x, gain, out, rows, d, eps);
   count_launch();
   return cudaGetLastError();
