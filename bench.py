@@ -31,6 +31,23 @@ DEFAULT_WORKLOAD = "cfg2_1p5b_b16"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+# DRAM bytes (read + write) of one gate/up GEMM launch of the default workload, from the ncu capture summarised in
+# profiles/gemm_f16_cfg2_4layers.md, and the hash of the kernel source that capture was taken with. A changed kernel
+# has no counters: traffic is then reported as null.
+GATEUP_TRAFFIC = {"workload": "cfg2_1p5b_b16", "bytes": 58.658816e6 + 4.5952e6,
+                  "source": "paper_2602_18447_b200/csrc/gemm_tcgen05.cu", "sha256_16": "4c41504f1f0eb3f6"}
+
+
+def gateup_traffic(workload: str):
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, GATEUP_TRAFFIC["source"]), "rb") as f:
+            h = hashlib.sha256(f.read()).hexdigest()[:16]
+    except OSError:
+        return None
+    return GATEUP_TRAFFIC["bytes"] if (workload == GATEUP_TRAFFIC["workload"] and h == GATEUP_TRAFFIC["sha256_16"]) else None
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -333,7 +350,8 @@ def run_ours(args, cfg):
         "roofline": {"kernel": "gemm_f16_kernel<256, SwiGLU> (gate/up projection)", "bound": "tensor",
                      "achieved": gu_tf, "peak": tensor_peak, "unit": "TFLOP/s", "frac": gu_tf / tensor_peak,
                      "peak_kind": f"{peak_kind} bf16 sustained (fp16 has the same nominal peak)",
-                     "traffic": None, "ms_per_launch": gu_ms, "launches_timed": prof["gemm_gateup"][1]},
+                     "traffic": (gateup_traffic(cfg.name) if args.layers is None else None), "traffic_unit": "bytes per launch (DRAM read + write, ncu)",
+                     "ms_per_launch": gu_ms, "launches_timed": prof["gemm_gateup"][1]},
         "kernels": kernels,
         "time_shares": shares,
     }
