@@ -342,11 +342,12 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   ap.status = m->status;
   const int plane_groups = kv->num_pages * d.n_kv_heads * kPageSize / 8;
 
+  const RopeEpilogue rope_epi{rope, d.head_dim / 2, (d.n_q_heads + d.n_kv_heads) * d.head_dim};
   for (int l = 0; l < d.n_layers; ++l) {
     const LayerDev& lw = m->layers[l];
     CS_STEP(kProfNorm, launch_rmsnorm(x, lw.norm1, a, T, d.d_model, d.rms_eps, s));
-    CS_STEP(kProfQkv, gemm_f16(tm_a, lw.tm_wqkv, nullptr, qkv, T, m->n_qkv, d.d_model, kEpiStoreF16, m->status, s));
-    CS_STEP(kProfRope, launch_rope_apply(qkv, rope, T, m->n_qkv, d.n_q_heads + d.n_kv_heads, d.head_dim, s));
+    // q and k heads leave the projection already rotated (the turn is applied to the fp32 accumulators)
+    CS_STEP(kProfQkv, gemm_f16_rope(tm_a, lw.tm_wqkv, qkv, T, m->n_qkv, d.d_model, rope_epi, m->status, s));
     ap.k_group_base = (2 * l) * plane_groups;
     ap.v_group_base = (2 * l + 1) * plane_groups;
     CS_STEP(kProfAttn, launch_attention(ap, kv->tm_pool, tm_qkv_attn, tm_q3d, d_items, L.n_items, s));

@@ -1,5 +1,5 @@
-// Memory-bound pieces of the decoder layers: embedding gather, RMSNorm, rotary tables and rotation,
-// and the scatter of K/V rows into cache pages.
+// Memory-bound pieces of the decoder layers: embedding gather, RMSNorm, rotary tables (the rotation itself is the
+// epilogue of the QKV projection), and the scatter of K/V rows into cache pages.
 #include "kernels.h"
 
 #include "common.cuh"
@@ -84,26 +84,6 @@ __global__ void rope_table_kernel(const int32_t* __restrict__ pos, const double*
   table[i] = make_float2(static_cast<float>(c), static_cast<float>(s));
 }
 
-// Thread per (row, head, pair of adjacent rotation pairs): elements j, j+1 and j+half, j+half+1.
-__global__ void rope_apply_kernel(uint16_t* __restrict__ qkv, const float2* __restrict__ table, int T, int n_qkv,
-                                  int n_rot_heads, int hd) {
-  const int half = hd >> 1;
-  const int per_row = n_rot_heads * (half >> 1);
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= T * per_row) return;
-  const int t = i / per_row;
-  const int r = i - t * per_row;
-  const int head = r / (half >> 1);
-  const int j = (r - head * (half >> 1)) * 2;
-  uint32_t* lo = reinterpret_cast<uint32_t*>(qkv + static_cast<size_t>(t) * n_qkv + head * hd + j);
-  uint32_t* hi = reinterpret_cast<uint32_t*>(qkv + static_cast<size_t>(t) * n_qkv + head * hd + half + j);
-  const uint32_t a = *lo, b = *hi;
-  const float2 cs0 = table[t * half + j], cs1 = table[t * half + j + 1];
-  const float2 av = unpack_f16x2(a), bv = unpack_f16x2(b);
-  *lo = pack_f16x2(av.x * cs0.x - bv.x * cs0.y, av.y * cs1.x - bv.y * cs1.y);
-  *hi = pack_f16x2(bv.x * cs0.x + av.x * cs0.y, bv.y * cs1.x + av.y * cs1.y);
-}
-
 // Thread per 16 bytes of a K row and of a V row.
 __global__ void kv_scatter_kernel(const uint16_t* __restrict__ src_k, const uint16_t* __restrict__ src_v,
                                   int row_stride, const int32_t* __restrict__ tok_seq,
@@ -182,15 +162,6 @@ cudaError_t launch_rope_table(const int32_t* pos, const double* inv_freq, float2
   if (T <= 0) return cudaSuccess;
   const int n = T * half;
   rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(pos, inv_freq, table, T, half);
-  count_launch();
-  return cudaGetLastError();
-}
-
-cudaError_t launch_rope_apply(uint16_t* qkv, const float2* table, int T, int n_qkv, int n_rot_heads, int hd,
-                              cudaStream_t s) {
-  if (T <= 0) return cudaSuccess;
-  const int n = T * n_rot_heads * (hd / 4);
-  rope_apply_kernel<<<(n + 255) / 256, 256, 0, s>>>(qkv, table, T, n_qkv, n_rot_heads, hd);
   count_launch();
   return cudaGetLastError();
 }

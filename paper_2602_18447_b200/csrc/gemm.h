@@ -10,7 +10,8 @@ namespace cs {
 enum GemmEpilogue {
   kEpiStoreF16 = 0,  // out fp16 [M,N] = a * w^T
   kEpiResidAdd = 1,   // out fp32 [M,N] += a * w^T   (atomic adds, k-range split over the SMs)
-  kEpiSwiGLU = 2      // out fp16 [M,N] = silu(a * w^T) * (a * w2^T)
+  kEpiSwiGLU = 2,     // out fp16 [M,N] = silu(a * w^T) * (a * w2^T)
+  kEpiStoreRope = 3   // out fp16 [M,N] = a * w^T with the rotary turn applied to the leading heads (QKV projection)
 };
 
 // 2D tensor map over a row-major [rows, cols] matrix of 16-bit floats (fp16, or bf16 for the kv cache);
@@ -36,6 +37,17 @@ bool make_kv_group_map(CUtensorMap* tm, const void* base, uint64_t rows, uint32_
 bool make_kv_rows_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t row_elems, uint32_t hd);
 // Tensor map of a GEMM operand ([rows, k] fp16, K-major): 128-row x 64-column boxes, 128-byte swizzle.
 bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k);
+
+// Rotary position turn fused into the store epilogue of the QKV projection: columns [0, n_rot_cols) are heads of
+// 2 * half columns in which the pair (j, j + half) of row t turns by the angle whose (cos, sin) is table[t * half + j];
+// the remaining columns (the V heads) are stored as they are. half is 32 or 64; N and n_rot_cols multiples of 2 * half.
+struct RopeEpilogue {
+  const float2* table;
+  int half;
+  int n_rot_cols;
+};
+cudaError_t gemm_f16_rope(const CUtensorMap& ta, const CUtensorMap& tb, void* out, int M, int N, int K,
+                          const RopeEpilogue& rope, uint32_t* status, cudaStream_t stream);
 
 cudaError_t gemm_f16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,
                       int K, int epilogue, uint32_t* status, cudaStream_t stream);

@@ -77,6 +77,15 @@ __device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.b
 __device__ __forceinline__ void st_shared_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(p)), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void st_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -115,7 +124,8 @@ template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                  const __grid_constant__ CUtensorMap tm_b2, const __grid_constant__ CUtensorMap tm_out,
-                 void* __restrict__ out, int M, int N, int m_tiles, int n_tiles, int kblocks, int total_units, int units_per_cta, uint32_t* status) {
+                 void* __restrict__ out, int M, int N, int m_tiles, int n_tiles, int kblocks, int total_units,
+                 int units_per_cta, const RopeEpilogue rope, uint32_t* status) {
   using L = GemmSmem<BN>;
   constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
   constexpr uint32_t kTmemCols = 2 * BN;
@@ -237,11 +247,19 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       const Segment sg = next_segment(u, end, kblocks);
       const int m0 = tile_m(sg.tile, m_tiles, n_tiles, EPI) * BM;
       const int n0 = tile_n(sg.tile, m_tiles, n_tiles, EPI) * OUT_BN;
+      const int row = m0 + quad * 32 + lane;
+      const bool row_ok = row < M;
+      // Rotary epilogue: this row's (cos, sin) pairs are fetched while the tile is still being accumulated.
+      float4 rot[32];
+      if (EPI == kEpiStoreRope && row_ok && n0 < rope.n_rot_cols) {
+        const float4* tb = reinterpret_cast<const float4*>(rope.table + static_cast<size_t>(row) * rope.half);
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (2 * j < rope.half) rot[j] = __ldg(tb + j);
+      }
       if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, status)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
-      const int row = m0 + quad * 32 + lane;
-      const bool row_ok = row < M;
       uint32_t r[32];
       if (EPI == kEpiSwiGLU) {
         uint32_t r2[32];
@@ -263,6 +281,54 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll
             for (int j = 0; j < 4; ++j)
               if (col + j * 8 < N) st_v4(o + col + j * 8, p[4 * j], p[4 * j + 1], p[4 * j + 2], p[4 * j + 3]);
+          }
+        }
+      } else if (EPI == kEpiStoreRope) {
+        __half* o = reinterpret_cast<__half*>(out) + static_cast<size_t>(row) * N;
+        const int hd = 2 * rope.half;
+#pragma unroll 1
+        for (int h0 = 0; h0 < BN && n0 + h0 < N; h0 += hd) {
+          if (n0 + h0 < rope.n_rot_cols) {
+            // pairs (j, j + half) of one head, 16 pairs at a time
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              if (c * 16 < rope.half) {
+                uint32_t lo[16], hi[16];
+                tmem_ld_32x16(t_row + h0 + c * 16, lo);
+                tmem_ld_32x16(t_row + h0 + rope.half + c * 16, hi);
+                tmem_ld_wait();
+                uint32_t plo[8], phi[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const float4 cs = rot[c * 8 + e];      // (cos, sin) of pairs 2e and 2e + 1 of this chunk
+                  const float a0 = __uint_as_float(lo[2 * e]), a1 = __uint_as_float(lo[2 * e + 1]);
+                  const float b0 = __uint_as_float(hi[2 * e]), b1 = __uint_as_float(hi[2 * e + 1]);
+                  plo[e] = pack_f16x2(a0 * cs.x - b0 * cs.y, a1 * cs.z - b1 * cs.w);
+                  phi[e] = pack_f16x2(b0 * cs.x + a0 * cs.y, b1 * cs.z + a1 * cs.w);
+                }
+                if (row_ok) {
+                  __half* ol = o + n0 + h0 + c * 16;
+                  st_v4(ol, plo[0], plo[1], plo[2], plo[3]);
+                  st_v4(ol + 8, plo[4], plo[5], plo[6], plo[7]);
+                  st_v4(ol + rope.half, phi[0], phi[1], phi[2], phi[3]);
+                  st_v4(ol + rope.half + 8, phi[4], phi[5], phi[6], phi[7]);
+                }
+              }
+            }
+          } else {
+#pragma unroll 1
+            for (int c = 0; c < hd / 32; ++c) {
+              tmem_ld_32x32(t_row + h0 + c * 32, r);
+              tmem_ld_wait();
+              if (row_ok) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  st_v4(o + n0 + h0 + c * 32 + j * 8, pack_f16x2(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1])),
+                        pack_f16x2(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3])),
+                        pack_f16x2(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5])),
+                        pack_f16x2(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7])));
+              }
+            }
           }
         }
       } else if (EPI == kEpiStoreF16) {
@@ -358,7 +424,7 @@ bool make_out_f32_map(CUtensorMap* tm, void* base, int rows, int cols) {
 
 template <int BN, int EPI>
 cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, void* out, int M, int N,
-                   int K, uint32_t* status, cudaStream_t stream) {
+                   int K, uint32_t* status, cudaStream_t stream, const RopeEpilogue& rope = RopeEpilogue{nullptr, 0, 0}) {
   using L = GemmSmem<BN>;
   constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
   static bool attr_set = false;
@@ -385,7 +451,7 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
   CUtensorMap tout = ta;   // only the residual epilogue reads it
   if (EPI == kEpiResidAdd && !make_out_f32_map(&tout, out, M, N)) return cudaErrorInvalidValue;
   gemm_f16_kernel<BN, EPI><<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tb, tb2, tout, out, M, N, m_tiles, n_tiles, kblocks, total,
-                                                                      upc, status);
+                                                                      upc, rope, status);
   count_launch();
   return cudaGetLastError();
 }
@@ -449,6 +515,14 @@ bool make_kv_rows_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t
 
 bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k) {
   return make_tensor_map_16b(tm, base, static_cast<uint64_t>(rows), static_cast<uint64_t>(k), 128, 64, true, false);
+}
+
+cudaError_t gemm_f16_rope(const CUtensorMap& ta, const CUtensorMap& tb, void* out, int M, int N, int K,
+                          const RopeEpilogue& rope, uint32_t* status, cudaStream_t stream) {
+  if (M <= 0) return cudaSuccess;
+  if (!rope.table || (rope.half != 32 && rope.half != 64) || N % (2 * rope.half) || rope.n_rot_cols % (2 * rope.half))
+    return cudaErrorInvalidValue;
+  return launch<256, kEpiStoreRope>(ta, tb, tb, out, M, N, K, status, stream, rope);
 }
 
 cudaError_t gemm_f16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,

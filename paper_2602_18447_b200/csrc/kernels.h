@@ -51,9 +51,6 @@ cudaError_t launch_rmsnorm(const float* x, const float* gain, uint16_t* out, int
 // cos/sin of pos[t] * inv_freq[j] in double, stored as float2 [T, half].
 cudaError_t launch_rope_table(const int32_t* pos, const double* inv_freq, float2* table, int T, int half,
                               cudaStream_t s);
-// Rotate the first n_rot_heads heads (q heads then k heads) of every row of qkv in place.
-cudaError_t launch_rope_apply(uint16_t* qkv, const float2* table, int T, int n_qkv, int n_rot_heads, int hd,
-                              cudaStream_t s);
 // Copy K and V rows into cache pages. src rows are [n_kv_heads*hd] wide at src_k/src_v + t*row_stride.
 // Row t goes to sequence tok_seq[t], position tok_pos[t]; when tok_seq is NULL, to sequence const_seq,
 // position pos0 + t. The cache holds bf16 values in the fp16 encoding: bf16 sources are re-encoded (exact in
