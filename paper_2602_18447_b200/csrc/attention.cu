@@ -552,9 +552,13 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       }
     } else if (it.n_splits > 1) {
       // ---- piece of a split key range: store the partial result, then the last piece to arrive combines them
+      // The partial O goes out as one bulk copy: every thread puts its row into the (now idle) K ring, 16-byte
+      // chunk c of row r at chunk position c ^ (r & 7) so that the writes do not collide on the banks, and one
+      // thread hands the [128][HD] block to the copy engine. The slot keeps that chunk order; the combining
+      // step undoes it.
+      uint8_t* stage = smem + L::kKOff;
       if (ok) {
         tc_fence_after();
-        float* po = p.part_o + (static_cast<size_t>(it.slot) * 128 + row) * HD;
 #pragma unroll 1
         for (int c = 0; c < HD / 32; ++c) {
           uint32_t o[32];
@@ -562,9 +566,19 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
           tmem_ld_wait();
 #pragma unroll
           for (int e = 0; e < 8; ++e)
-            __stcg(reinterpret_cast<uint4*>(po + c * 32 + e * 4), make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]));
+            *reinterpret_cast<uint4*>(stage + row * (HD * 4) + (((c * 8 + e) ^ (row & 7)) << 4)) =
+                make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
         }
         __stcg(reinterpret_cast<float2*>(p.part_ml + (static_cast<size_t>(it.slot) * 128 + row) * 2), make_float2(m_ref, l));
+        fence_proxy_async();
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ok && warp == 2 && lane == 0) {
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     ::"l"(p.part_o + static_cast<size_t>(it.slot) * 128 * HD), "r"(smem_u32(stage)), "r"(128 * HD * 4)
+                     : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
       }
       __threadfence();
       asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -609,7 +623,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
                 v[ss][rr] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (s0 + ss < it.n_splits && lane < kLanes)
                   v[ss][rr] = __ldcg(reinterpret_cast<const float4*>(
-                      p.part_o + (static_cast<size_t>(it.slot0 + s0 + ss) * 128 + r) * HD + lane * kColsPerLane));
+                      p.part_o + (static_cast<size_t>(it.slot0 + s0 + ss) * 128 + r) * HD + ((lane ^ (r & 7)) << 2)));
               }
 #pragma unroll
             for (int ss = 0; ss < 4; ++ss)
