@@ -318,6 +318,9 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_slot;
+  // Set-up overlapped the previous kernel's tail; q, k, v of the new tokens are needed from here on.
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp == 0 || warp == 6) {
     // ------------------------------------------------------------ TMA producers (whole warps): warp 0 K, warp 6 V
@@ -671,9 +674,10 @@ cudaError_t launch_hd(const AttnParams& p, const CUtensorMap& tm_pool, const CUt
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  attention_kernel<HD><<<n_items, kAttnThreads, L::kTotal, s>>>(p, tm_pool, tm_kv_new, tm_q3d, items);
+  cudaError_t le = launch_pdl(attention_kernel<HD>, dim3(n_items), dim3(kAttnThreads), L::kTotal, s, p, tm_pool, tm_kv_new, tm_q3d,
+                              items);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace

@@ -30,6 +30,15 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of the pass is launched with programmatic stream serialisation: its CTAs may be scheduled while the
+// previous kernel is still draining, so that launch latency and set-up (barriers, tensor memory, descriptor
+// fetches) overlap the previous kernel's tail. pdl_wait() returns once the previous kernel has completed and its
+// writes are visible; nothing that another kernel of the pass writes may be touched before it, and every thread
+// calls it before it exits, so that "this kernel has completed" always implies "its predecessors have".
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));

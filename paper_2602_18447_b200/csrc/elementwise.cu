@@ -12,6 +12,8 @@ thread_local int64_t g_launches = 0;
 
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const uint16_t* __restrict__ embed,
                              float* __restrict__ x, int T, int d, int vocab) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int t = blockIdx.x;
   int tok = tokens[t];
   tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);
@@ -30,6 +32,8 @@ constexpr int kNormRegVecs = 32;   // float4 per lane
 
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
                                uint16_t* __restrict__ out, int rows, int d, float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
@@ -76,6 +80,8 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
 
 __global__ void rope_table_kernel(const int32_t* __restrict__ pos, const double* __restrict__ inv_freq,
                                   float2* __restrict__ table, int T, int half) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= T * half) return;
   const int t = i / half, j = i - t * half;
@@ -91,6 +97,8 @@ __global__ void kv_scatter_kernel(const uint16_t* __restrict__ src_k, const uint
                                   const int32_t* __restrict__ page_table,
                                   int max_pages_per_seq, uint16_t* __restrict__ pool_k, uint16_t* __restrict__ pool_v,
                                   int n_kv_heads, int hd, int page_size, int T, int src_is_f16) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int chunks = n_kv_heads * hd / 8;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= T * chunks) return;
@@ -143,27 +151,27 @@ int64_t take_launch_count() {
 cudaError_t launch_embed(const int32_t* tokens, const uint16_t* embed, float* x, int T, int d, int vocab,
                          cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
-  embed_kernel<<<T, 128, 0, s>>>(tokens, embed, x, T, d, vocab);
+  cudaError_t le = launch_pdl(embed_kernel, dim3(T), dim3(128), 0, s, tokens, embed, x, T, d, vocab);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 cudaError_t launch_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps,
                            cudaStream_t s) {
   if (rows <= 0) return cudaSuccess;
   const int warps = 4;
-  rmsnorm_kernel<<<(rows + warps - 1) / warps, warps * 32, 0, s>>>(x, gain, out, rows, d, eps);
+  cudaError_t le = launch_pdl(rmsnorm_kernel, dim3((rows + warps - 1) / warps), dim3(warps * 32), 0, s, x, gain, out, rows, d, eps);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 cudaError_t launch_rope_table(const int32_t* pos, const double* inv_freq, float2* table, int T, int half,
                               cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   const int n = T * half;
-  rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(pos, inv_freq, table, T, half);
+  cudaError_t le = launch_pdl(rope_table_kernel, dim3((n + 255) / 256), dim3(256), 0, s, pos, inv_freq, table, T, half);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int row_stride, const int32_t* tok_seq,

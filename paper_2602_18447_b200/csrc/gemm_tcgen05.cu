@@ -170,6 +170,9 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above overlapped the previous kernel's tail; its results (the A operand, x) are needed from here on.
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -450,10 +453,10 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
   }
   CUtensorMap tout = ta;   // only the residual epilogue reads it
   if (EPI == kEpiResidAdd && !make_out_f32_map(&tout, out, M, N)) return cudaErrorInvalidValue;
-  gemm_f16_kernel<BN, EPI><<<grid, kGemmThreads, L::kTotal, stream>>>(ta, tb, tb2, tout, out, M, N, m_tiles, n_tiles, kblocks, total,
-                                                                      upc, rope, status);
+  cudaError_t le = launch_pdl(gemm_f16_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), L::kTotal, stream, ta, tb, tb2, tout, out, M,
+                              N, m_tiles, n_tiles, kblocks, total, upc, rope, status);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace

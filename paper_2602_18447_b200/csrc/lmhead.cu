@@ -94,6 +94,8 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -223,6 +225,8 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
 __global__ void last_rows_norm_kernel(const float* __restrict__ x, const int32_t* __restrict__ cu_new,
                                       const float* __restrict__ gain, uint16_t* __restrict__ h, int B, int B_pad,
                                       int d, float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (b >= B_pad) return;
@@ -252,6 +256,8 @@ __global__ void gate_kernel(const float* __restrict__ part_max, const float* __r
                             int nb_stride, const float* __restrict__ verdict_logits, int n_verdict, int B, float tau,
                             float* __restrict__ out_conf, uint8_t* __restrict__ out_accept,
                             int32_t* __restrict__ out_verdict, float* __restrict__ out_lse) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (b >= B) return;
@@ -325,9 +331,9 @@ cudaError_t launch_lm_nb(const CUtensorMap& tm_w, const CUtensorMap& tm_h, const
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  lm_head_kernel<NB><<<grid, kLmThreads, L::kTotal, s>>>(tm_w, tm_h, a);
+  cudaError_t le = launch_pdl(lm_head_kernel<NB>, dim3(grid), dim3(kLmThreads), L::kTotal, s, tm_w, tm_h, a);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace
