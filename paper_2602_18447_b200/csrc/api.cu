@@ -160,10 +160,11 @@ struct BatchLayout {
 // Cost of an attention work item in key tiles: the tiles themselves plus the fixed part of a CTA (set-up, Q load,
 // pipeline fill, epilogue), what being a piece of a split query tile adds (the partial result goes through global
 // memory), and what the last piece adds by combining the partial results.
-// Measured on B200: a tile takes ~2 k cycles; set-up to first S ~5.5 k; the epilogue of a piece (partial store,
-// fence, counter) ~7 k against ~1.5 k for a whole range.
+// Measured on B200: a tile takes ~2 k cycles; set-up to first S ~5.5 k; the epilogue of a piece (partial block out
+// by bulk copy, fence, counter) ~5 k against ~1.5 k for a whole range; the combining piece fetches all blocks in one
+// round of bulk copies.
 constexpr double kAttnItemFixed = 3.5;
-constexpr double kAttnPieceExtra = 3.0;
+constexpr double kAttnPieceExtra = 2.0;
 constexpr double kAttnMergeFixed = 1.0;
 constexpr double kAttnMergePerSplit = 0.5;
 
@@ -222,13 +223,17 @@ void build_attention_work(const cs_model* m, int B, const int32_t* lens, const i
   };
   int best_cap = longest;
   double best = estimate(longest);
-  // Only caps that cut most query tiles are tried: cutting just the few longest ones in two was measured slower
-  // than leaving the batch whole (29 -> 37 us at batch 16), a piece costs more than its share of the tiles.
-  for (int k = 2; k <= 16 && longest / k >= 2; ++k) {
-    const int cap = (longest + k - 1) / k;
+  int last_cap = longest;
+  auto consider = [&](int cap) {
+    if (cap < 2 || cap >= last_cap) return;
+    last_cap = cap;
     const double e = estimate(cap);
     if (e < 0.97 * best) { best = e; best_cap = cap; }
-  }
+  };
+  // caps just below the longest range cut only the few longest query tiles (in two) ...
+  for (int pct = 92; pct >= 52; pct -= 8) consider((longest * pct + 99) / 100);
+  // ... smaller ones cut most of them, into more pieces
+  for (int k = 2; k <= 16; ++k) consider((longest + k - 1) / k);
   items.clear();
   int slots = 0;
   for (const Unit& u : units)

@@ -258,6 +258,7 @@ struct Bars {
   uint64_t pv_done[kSBufs];                     // P V complete
   uint32_t tmem_slot;
   uint32_t abort_flag;
+  uint64_t merge_bar;                           // partial blocks of a round have landed (combining piece only)
   uint32_t is_last;
 };
 
@@ -281,6 +282,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_full, 1);
+    mbar_init(&bars->merge_bar, 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&bars->k_full[s], 1);
       mbar_init(&bars->k_empty[s], 1);
@@ -597,60 +599,53 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (bars->is_last) {
         __threadfence();
-        // Each warp combines its 32 rows, four rows at a time; within a row the lanes split the columns.
-        constexpr int kColsPerLane = 4;
-        constexpr int kLanes = HD / kColsPerLane;   // 32 for HD 128, 16 for HD 64
-        for (int r0 = 0; r0 < 32; r0 += 4) {
-          float wgt[4], inv[4];
+        // Combine the pieces. Their partial O blocks are fetched into the idle K/V rings by bulk copies, as many
+        // per round as fit, so that the whole round costs one trip to L2; then every thread combines its own row
+        // from shared memory. (Reading the blocks from global memory a few rows at a time took ~15 k cycles.)
+        constexpr int kBlockBytes = 128 * HD * 4;
+        constexpr int kPerRound = (2 * kStages * L::kTileBytes) / kBlockBytes;
+        float mmax = -INFINITY;
+        for (int sp = 0; sp < it.n_splits; ++sp)
+          mmax = fmaxf(mmax, __ldcg(p.part_ml + (static_cast<size_t>(it.slot0 + sp) * 128 + row) * 2));
+        float acc[HD];
 #pragma unroll
-          for (int rr = 0; rr < 4; ++rr) {
-            const int r = quad * 32 + r0 + rr;
-            float2 ml = make_float2(-INFINITY, 0.f);
-            if (lane < it.n_splits)
-              ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (static_cast<size_t>(it.slot0 + lane) * 128 + r) * 2));
-            const float mmax = warp_max(ml.x);
-            const float w = (ml.x == -INFINITY) ? 0.f : fast_exp2((ml.x - mmax) * sc);
-            wgt[rr] = w;
-            inv[rr] = 1.f / warp_sum(w * ml.y);
+        for (int e = 0; e < HD; ++e) acc[e] = 0.f;
+        float lsum = 0.f;
+        uint32_t round = 0;
+        for (int s0 = 0; s0 < it.n_splits && ok; s0 += kPerRound, ++round) {
+          const int cnt = min(kPerRound, it.n_splits - s0);
+          if (warp == 2 && lane == 0) {
+            mbar_arrive_expect_tx(&bars->merge_bar, static_cast<uint32_t>(cnt) * kBlockBytes);
+            for (int i = 0; i < cnt; ++i)
+              asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                           ::"r"(smem_u32(stage + i * kBlockBytes)),
+                             "l"(p.part_o + static_cast<size_t>(it.slot0 + s0 + i) * 128 * HD), "r"(kBlockBytes),
+                             "r"(smem_u32(&bars->merge_bar))
+                           : "memory");
           }
-          float4 acc[4];
+          if (!mbar_wait(&bars->merge_bar, round & 1u, abort_flag, p.status)) { ok = false; break; }
+          for (int i = 0; i < cnt; ++i) {
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (static_cast<size_t>(it.slot0 + s0 + i) * 128 + row) * 2));
+            if (ml.x == -INFINITY) continue;
+            const float w = fast_exp2((ml.x - mmax) * sc);
+            lsum += w * ml.y;
+            const uint8_t* src = stage + i * kBlockBytes + row * (HD * 4);
 #pragma unroll
-          for (int rr = 0; rr < 4; ++rr) acc[rr] = make_float4(0.f, 0.f, 0.f, 0.f);
-          for (int s0 = 0; s0 < it.n_splits; s0 += 4) {
-            float4 v[4][4];
-#pragma unroll
-            for (int ss = 0; ss < 4; ++ss)
-#pragma unroll
-              for (int rr = 0; rr < 4; ++rr) {
-                const int r = quad * 32 + r0 + rr;
-                v[ss][rr] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (s0 + ss < it.n_splits && lane < kLanes)
-                  v[ss][rr] = __ldcg(reinterpret_cast<const float4*>(
-                      p.part_o + (static_cast<size_t>(it.slot0 + s0 + ss) * 128 + r) * HD + ((lane ^ (r & 7)) << 2)));
-              }
-#pragma unroll
-            for (int ss = 0; ss < 4; ++ss)
-#pragma unroll
-              for (int rr = 0; rr < 4; ++rr) {
-                const float w = __shfl_sync(0xffffffffu, wgt[rr], (s0 + ss) & 31);
-                if (s0 + ss < it.n_splits && w != 0.f) {
-                  acc[rr].x += w * v[ss][rr].x; acc[rr].y += w * v[ss][rr].y;
-                  acc[rr].z += w * v[ss][rr].z; acc[rr].w += w * v[ss][rr].w;
-                }
-              }
-          }
-#pragma unroll
-          for (int rr = 0; rr < 4; ++rr) {
-            const int r = quad * 32 + r0 + rr;
-            const int pl = r / G;
-            const int ps = it.q_tok0 + pl;
-            if (pl < ntok && ps < n_new && lane < kLanes) {
-              uint16_t* dst = p.out + static_cast<size_t>(tok0 + ps) * q_dim + (it.kv_head * G + (r - pl * G)) * HD +
-                              lane * kColsPerLane;
-              *reinterpret_cast<uint2*>(dst) = make_uint2(pack_f16x2(acc[rr].x * inv[rr], acc[rr].y * inv[rr]),
-                                                          pack_f16x2(acc[rr].z * inv[rr], acc[rr].w * inv[rr]));
+            for (int c = 0; c < HD / 4; ++c) {
+              const float4 v = *reinterpret_cast<const float4*>(src + ((c ^ (row & 7)) << 4));
+              acc[4 * c] += w * v.x; acc[4 * c + 1] += w * v.y; acc[4 * c + 2] += w * v.z; acc[4 * c + 3] += w * v.w;
             }
           }
+          asm volatile("bar.sync 1, 128;" ::: "memory");     // the next round overwrites the blocks
+        }
+        if (ok && row_ok) {
+          const float inv = 1.f / lsum;
+          uint16_t* dst = p.out + static_cast<size_t>(tok0 + pos) * q_dim + (it.kv_head * G + g) * HD;
+#pragma unroll
+          for (int c = 0; c < HD / 8; ++c)
+            *reinterpret_cast<uint4*>(dst + c * 8) = make_uint4(
+                pack_f16x2(acc[8 * c] * inv, acc[8 * c + 1] * inv), pack_f16x2(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv),
+                pack_f16x2(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv), pack_f16x2(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv));
         }
       }
     }
