@@ -23,8 +23,9 @@ Parity pins (tests/test_oracle_*.py): closed forms for each block, brute-force
 attention with scalar loops, cache-extend == full causal recompute, rotary
 shift invariance, GQA == MHA with repeated heads, softmax sums to one, gate
 end points of Table 3 (gamma = 0 never escalates, gamma > 1 always does),
-batch-permutation equivariance, and the whole forward against the
-`transformers` Qwen2 architecture used as a black-box library routine.
+batch-permutation equivariance, the whole forward against the
+`transformers` Qwen2 architecture used as a black-box library routine, and hand-worked iterations of
+Algorithm 1 / Eq. 5 for the selection bookkeeping (tests/golden/cascade_cases.txt).
 """
 from __future__ import annotations
 
@@ -177,6 +178,50 @@ def escalate_list(conf: np.ndarray, tau: float) -> Tuple[np.ndarray, np.ndarray,
     acc = gate(conf, tau)
     idx = np.nonzero(acc == 0)[0].astype(np.int32)
     return acc, idx, int(idx.shape[0])
+
+
+def cascade_select(trusted: Sequence[int], verdict_d: Sequence[int], conf_d: Sequence[float],
+                   verdict_t: Optional[Sequence[int]], conf_t: Optional[Sequence[float]],
+                   req_offsets: Sequence[int], accept_index: int = 0
+                   ) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """What the drafting loop does with the verification results of one iteration, per request (the steps of
+    request r are [req_offsets[r], req_offsets[r+1]) of the batch).
+
+    Final decision of a step (Algorithm 1, Stage 2; Eq. 4): the draft verifier's decision r_D when it was
+    trusted (p_D >= gamma), else the target verifier's decision; a step that was escalated but has no target
+    result counts as rejected. Its confidence is that of the verifier whose decision was taken (Section 4.3).
+    Linear drafting (Algorithm 1, the loop over j with `break`): m = number of leading steps of the request
+    whose final decision is "accept". Tree drafting (Section 4.3, Eq. 5): among the request's candidates that
+    pass verification, the one with the highest confidence (the earliest on ties); -1 if none passes.
+
+    Returns (passed uint8 [B], final confidence float32 [B], m int32 [R], best int32 [R] batch index or -1).
+    Written as plain loops: this is bookkeeping, not arithmetic."""
+    B = len(trusted)
+    passed = np.zeros(B, dtype=np.uint8)
+    conf = np.zeros(B, dtype=np.float32)
+    for i in range(B):
+        if trusted[i]:
+            passed[i] = 1 if verdict_d[i] == accept_index else 0
+            conf[i] = np.float32(conf_d[i])
+        elif verdict_t is not None:
+            passed[i] = 1 if verdict_t[i] == accept_index else 0
+            conf[i] = np.float32(conf_t[i])
+        else:
+            passed[i] = 0
+            conf[i] = np.float32(conf_d[i])
+    R = len(req_offsets) - 1
+    m = np.zeros(R, dtype=np.int32)
+    best = np.full(R, -1, dtype=np.int32)
+    for r in range(R):
+        lo, hi = int(req_offsets[r]), int(req_offsets[r + 1])
+        j = lo
+        while j < hi and passed[j]:
+            j += 1
+        m[r] = j - lo
+        for i in range(lo, hi):
+            if passed[i] and not np.isnan(conf[i]) and (best[r] < 0 or conf[i] > conf[best[r]]):
+                best[r] = i
+    return passed, conf, m, best
 
 
 # ----------------------------------------------------------------------------------------------

@@ -221,3 +221,34 @@ def test_escalate_list_is_complement_in_order():
     assert acc.tolist() == [1, 0, 1, 0, 0] and idx.tolist() == [1, 3, 4] and cnt == 3
     acc, idx, cnt = O.escalate_list(conf, 0.0)
     assert cnt == 0 and idx.shape == (0,)
+
+
+def test_cascade_select_hand_worked_iterations():
+    """Algorithm 1's sequential accept loop and Eq. 5's choice, against cases worked by hand."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "cascade_cases.txt")
+    rows = [l for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(rows) >= 8
+    trusted, vd, cd, vt, ct, offs, want_m, want_best = [], [], [], [], [], [0], [], []
+    for line in rows:
+        steps, exp = line.split("|")
+        for tok in steps.split():
+            t, dec, p = tok[0] == "T", 0 if tok[1] == "a" else 1, float(tok[2:])
+            trusted.append(1 if t else 0)
+            # the verifier that does not count says the opposite with another confidence: it must be ignored
+            vd.append(dec if t else 1 - dec); cd.append(p if t else 0.123)
+            vt.append(dec if not t else 1 - dec); ct.append(p if not t else 0.999)
+        m, best = exp.split()
+        want_m.append(int(m))
+        want_best.append(-1 if int(best) < 0 else offs[-1] + int(best))
+        offs.append(len(trusted))
+    passed, conf, m, best = O.cascade_select(trusted, vd, cd, vt, ct, offs, accept_index=0)
+    assert m.tolist() == want_m and best.tolist() == want_best
+    # invariants: m never exceeds the request's length; all accepted -> m = length; best is an accepted step
+    for r in range(len(want_m)):
+        k = offs[r + 1] - offs[r]
+        assert 0 <= m[r] <= k and (m[r] == k) == bool(passed[offs[r]:offs[r + 1]].all())
+        assert best[r] == -1 or passed[best[r]]
+    # without target results every escalated step is a rejection
+    p2, _, m2, _ = O.cascade_select(trusted, vd, cd, None, None, offs)
+    assert all(p2[i] == 0 for i in range(len(trusted)) if not trusted[i]) and np.all(m2 <= m)
