@@ -180,6 +180,28 @@ int cs_escalate_mask(const float* conf, int B, float tau, uint8_t* out_accept,
                      int32_t* out_escalate_idx, int32_t* out_escalate_count, void* stream);
 
 /*
+ * cs_cascade_select - what the drafting loop does with the verification results of one iteration, on the device.
+ * Final decision of step i (Algorithm 1, Stage 2; Eq. 4): the draft verifier's decision when it was trusted
+ * (trusted[i] != 0, i.e. p_D >= gamma), else the target verifier's; an escalated step without a target result
+ * (verdict_t == NULL) counts as rejected. Its confidence is that of the verifier whose decision was taken.
+ * Per request r, whose steps are [req_offsets[r], req_offsets[r+1]) of the batch:
+ *   out_prefix_len[r]  m of Algorithm 1: the number of leading steps whose final decision is "accept" (the loop
+ *                      over the drafted steps breaks at the first rejection);
+ *   out_best[r]        tree drafting (Section 4.3, Eq. 5): batch index of the accepted candidate with the highest
+ *                      confidence, the earliest on ties, or -1 if none was accepted.
+ *   trusted            device uint8[B]  (out_accept of the draft pass).
+ *   verdict_d, conf_d  device int32[B], float[B] (out_verdict, out_conf of the draft pass).
+ *   verdict_t, conf_t  device int32[B], float[B], read only where trusted[i] == 0, or both NULL.
+ *   req_offsets        device int32[R+1], ascending, req_offsets[0] .. req_offsets[R] within [0, B].
+ *   accept_index       which entry of verdict_ids means "accept" (0..7).
+ *   out_pass, out_conf device uint8[B], float[B] or NULL: the final decision (1 = accept) and confidence per step.
+ * Asynchronous on `stream`. Errors: CS_EINVAL.
+ */
+int cs_cascade_select(const uint8_t* trusted, const int32_t* verdict_d, const float* conf_d, const int32_t* verdict_t,
+                      const float* conf_t, const int32_t* req_offsets, int R, int accept_index, int32_t* out_prefix_len,
+                      int32_t* out_best, uint8_t* out_pass, float* out_conf, void* stream);
+
+/*
  * Debug / test access. cs_set_keep_logits(model, 1) makes every later cs_verify_steps also write the full
  * last-position logits (fp32 [B, vocab]) into the workspace; cs_get_last_logits copies them to
  * dev_out (device float[B*vocab]) on `stream`. cs_get_last_lse copies the per-step logsumexp

@@ -16,7 +16,7 @@ CS_OK, CS_EINVAL, CS_ENOMEM, CS_ECUDA, CS_ETIMEOUT, CS_ESTATE, CS_ELIMIT = range
 EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_reserve",
     "cs_kv_alloc", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
-    "cs_verify_steps", "cs_escalate_mask", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
+    "cs_verify_steps", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
     "cs_last_status", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_profile", "cs_profile_read",
 ]
 
@@ -74,6 +74,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_prefill": (C.c_int, [vp, vp, vp, vp, vp, i32, vp]),
         "cs_verify_steps": (C.c_int, [vp, vp, vp, i32, vp, i32, vp, vp, i32, f32, vp, vp, vp, vp]),
         "cs_escalate_mask": (C.c_int, [vp, i32, f32, vp, vp, vp, vp]),
+        "cs_cascade_select": (C.c_int, [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]),
         "cs_set_keep_logits": (C.c_int, [vp, i32]),
         "cs_get_last_logits": (C.c_int, [vp, vp, i32, vp]),
         "cs_get_last_lse": (C.c_int, [vp, vp, i32, vp]),
@@ -231,6 +232,16 @@ def cs_escalate_mask(conf, tau: float, out_accept, out_escalate_idx, out_escalat
     _check(load_library().cs_escalate_mask(_dev_ptr(conf), int(conf.shape[0]), float(tau), _dev_ptr(out_accept),
                                            _dev_ptr(out_escalate_idx), _dev_ptr(out_escalate_count),
                                            _stream_ptr(stream)), "cs_escalate_mask")
+
+
+def cs_cascade_select(trusted, verdict_d, conf_d, verdict_t, conf_t, req_offsets, accept_index: int, out_prefix_len,
+                      out_best, out_pass=None, out_conf=None, stream=None) -> None:
+    """All arguments are CUDA tensors (verdict_t / conf_t / out_pass / out_conf may be None); req_offsets int32 [R+1]."""
+    _check(load_library().cs_cascade_select(_dev_ptr(trusted), _dev_ptr(verdict_d), _dev_ptr(conf_d), _dev_ptr(verdict_t),
+                                            _dev_ptr(conf_t), _dev_ptr(req_offsets), int(req_offsets.shape[0]) - 1,
+                                            int(accept_index), _dev_ptr(out_prefix_len), _dev_ptr(out_best),
+                                            _dev_ptr(out_pass), _dev_ptr(out_conf), _stream_ptr(stream)),
+           "cs_cascade_select")
 
 
 def cs_set_keep_logits(model: int, keep: bool) -> None:

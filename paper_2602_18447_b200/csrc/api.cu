@@ -804,6 +804,18 @@ int cs_escalate_mask(const float* conf, int B, float tau, uint8_t* out_accept, i
   return CS_OK;
 }
 
+int cs_cascade_select(const uint8_t* trusted, const int32_t* verdict_d, const float* conf_d, const int32_t* verdict_t,
+                      const float* conf_t, const int32_t* req_offsets, int R, int accept_index, int32_t* out_prefix_len,
+                      int32_t* out_best, uint8_t* out_pass, float* out_conf, void* stream) {
+  if (R < 0 || accept_index < 0 || accept_index > 7) return CS_EINVAL;
+  if (R == 0) return CS_OK;
+  if (!trusted || !verdict_d || !conf_d || !req_offsets || !out_prefix_len || !out_best) return CS_EINVAL;
+  if ((verdict_t == nullptr) != (conf_t == nullptr)) return CS_EINVAL;
+  CS_CUDA(launch_cascade_select(trusted, verdict_d, conf_d, verdict_t, conf_t, req_offsets, R, accept_index,
+                                out_prefix_len, out_best, out_pass, out_conf, static_cast<cudaStream_t>(stream)));
+  return CS_OK;
+}
+
 int cs_set_keep_logits(cs_model* m, int keep) {
   if (!m) return CS_EINVAL;
   m->keep_logits = keep != 0;

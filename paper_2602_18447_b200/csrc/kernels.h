@@ -86,6 +86,10 @@ int lm_head_batch_pad(int B);
 cudaError_t launch_gate(const float* part_max, const float* part_sum, int n_slices, int nb_stride,
                         const float* verdict_logits, int n_verdict, int B, float tau, float* out_conf,
                         uint8_t* out_accept, int32_t* out_verdict, float* out_lse, cudaStream_t s);
+cudaError_t launch_cascade_select(const uint8_t* trusted, const int32_t* verdict_d, const float* conf_d,
+                                  const int32_t* verdict_t, const float* conf_t, const int32_t* req_offsets, int R,
+                                  int accept_index, int32_t* out_prefix_len, int32_t* out_best, uint8_t* out_pass,
+                                  float* out_conf, cudaStream_t s);
 cudaError_t launch_escalate(const float* conf, int B, float tau, uint8_t* out_accept, int32_t* out_idx,
                             int32_t* out_count, cudaStream_t s);
 

@@ -322,6 +322,59 @@ __global__ void escalate_kernel(const float* __restrict__ conf, int B, float tau
   if (threadIdx.x == 0) *out_count = base;
 }
 
+// One warp per request: final decision and confidence of each of its steps (Eq. 4), the length of the leading run
+// of accepted steps (Algorithm 1's loop with break) and the accepted step with the highest confidence (Eq. 5).
+__global__ void cascade_select_kernel(const uint8_t* __restrict__ trusted, const int32_t* __restrict__ verdict_d,
+                                      const float* __restrict__ conf_d, const int32_t* __restrict__ verdict_t,
+                                      const float* __restrict__ conf_t, const int32_t* __restrict__ req_offsets, int R,
+                                      int accept_index, int32_t* __restrict__ out_prefix_len,
+                                      int32_t* __restrict__ out_best, uint8_t* __restrict__ out_pass,
+                                      float* __restrict__ out_conf) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (r >= R) return;
+  const int lo = req_offsets[r], hi = req_offsets[r + 1];
+  int prefix = -1;                       // first rejected position, once found
+  float best_c = -INFINITY;
+  int best_i = -1;
+  for (int i0 = lo; i0 < hi; i0 += 32) {
+    const int i = i0 + lane;
+    bool pass = false;
+    float c = 0.f;
+    if (i < hi) {
+      if (trusted[i]) {
+        pass = verdict_d[i] == accept_index;
+        c = conf_d[i];
+      } else if (verdict_t) {
+        pass = verdict_t[i] == accept_index;
+        c = conf_t[i];
+      } else {
+        c = conf_d[i];
+      }
+      if (out_pass) out_pass[i] = pass ? 1 : 0;
+      if (out_conf) out_conf[i] = c;
+    }
+    const unsigned rejected = __ballot_sync(0xffffffffu, i < hi && !pass);
+    if (prefix < 0 && rejected) prefix = i0 - lo + (__ffs(rejected) - 1);
+    // highest confidence among the accepted steps, the earliest on ties (NaN never wins)
+    float cand = (i < hi && pass && c == c) ? c : -INFINITY;
+    int idx = (cand > -INFINITY) ? i : 0x7fffffff;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float oc = __shfl_xor_sync(0xffffffffu, cand, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+      if (oc > cand || (oc == cand && oi < idx)) { cand = oc; idx = oi; }
+    }
+    if (idx != 0x7fffffff && (best_i < 0 || cand > best_c)) { best_c = cand; best_i = idx; }
+  }
+  if (lane == 0) {
+    out_prefix_len[r] = prefix < 0 ? hi - lo : prefix;
+    out_best[r] = best_i;
+  }
+}
+
 template <int NB>
 cudaError_t launch_lm_nb(const CUtensorMap& tm_w, const CUtensorMap& tm_h, const LmArgs& a, int grid, cudaStream_t s) {
   using L = LmSmem<NB>;
@@ -388,6 +441,19 @@ cudaError_t launch_gate(const float* part_max, const float* part_sum, int n_slic
   gate_kernel<<<(B + warps - 1) / warps, warps * 32, 0, s>>>(part_max, part_sum, n_slices, nb_stride, verdict_logits,
                                                            n_verdict, B, tau, out_conf, out_accept, out_verdict,
                                                            out_lse);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_cascade_select(const uint8_t* trusted, const int32_t* verdict_d, const float* conf_d,
+                                  const int32_t* verdict_t, const float* conf_t, const int32_t* req_offsets, int R,
+                                  int accept_index, int32_t* out_prefix_len, int32_t* out_best, uint8_t* out_pass,
+                                  float* out_conf, cudaStream_t s) {
+  if (R <= 0) return cudaSuccess;
+  const int warps = 4;
+  cascade_select_kernel<<<(R + warps - 1) / warps, warps * 32, 0, s>>>(trusted, verdict_d, conf_d, verdict_t, conf_t,
+                                                                     req_offsets, R, accept_index, out_prefix_len,
+                                                                     out_best, out_pass, out_conf);
   count_launch();
   return cudaGetLastError();
 }

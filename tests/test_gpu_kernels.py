@@ -131,3 +131,36 @@ def test_lm_head_gate_matches_oracle(B, d, vocab):
         assert np.array_equal(out_v.cpu().numpy()[clear], verdict[clear])
     if B > 4:
         assert 0 < (conf >= 0.3).sum() < B
+
+
+def test_cascade_select_matches_oracle_bit_exact():
+    """Algorithm 1's accept-prefix length and Eq. 5's choice per request, on random iterations: requests of 0 to 70
+    steps (more than one warp's worth), ties in the confidence, NaN confidences, with and without target results."""
+    import torch
+    from paper_2602_18447_b200 import binding as B
+    g = np.random.default_rng(77)
+    for trial in range(6):
+        sizes = g.integers(0, 12, size=40).tolist() + [70, 33, 1, 0, 32]
+        offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+        n = int(offs[-1])
+        trusted = (g.uniform(size=n) < 0.6).astype(np.uint8)
+        vd = (g.uniform(size=n) < 0.25).astype(np.int32)
+        vt = (g.uniform(size=n) < 0.4).astype(np.int32)
+        cd = np.round(g.uniform(0.5, 1.0, size=n), 1).astype(np.float32)     # coarse grid: many ties
+        ct = np.round(g.uniform(0.5, 1.0, size=n), 1).astype(np.float32)
+        cd[::17] = np.nan
+        with_target = trial % 2 == 0
+        want = O.cascade_select(trusted, vd, cd, vt if with_target else None, ct if with_target else None, offs, 0)
+        dev = lambda a: torch.from_numpy(a).cuda()
+        R = len(sizes)
+        m = torch.full((R,), -7, dtype=torch.int32, device="cuda")
+        best = torch.full((R,), -7, dtype=torch.int32, device="cuda")
+        passed = torch.full((n,), 9, dtype=torch.uint8, device="cuda")
+        conf = torch.full((n,), -1.0, dtype=torch.float32, device="cuda")
+        B.cs_cascade_select(dev(trusted), dev(vd), dev(cd), dev(vt) if with_target else None,
+                            dev(ct) if with_target else None, dev(offs), 0, m, best, passed, conf)
+        torch.cuda.synchronize()
+        assert np.array_equal(passed.cpu().numpy(), want[0])
+        assert np.array_equal(conf.cpu().numpy(), want[1], equal_nan=True)
+        assert np.array_equal(m.cpu().numpy(), want[2])
+        assert np.array_equal(best.cpu().numpy(), want[3])
