@@ -20,6 +20,8 @@ def weights_1p5b():
 
 def _run_full(name, weights, sample):
     cfg = get_config(name)
+    if weights is None:
+        weights = model_weights(cfg.model, cfg.seed)
     batch = make_batch(cfg)
     ses = P.build_session(cfg, weights, batch)
     try:
@@ -72,3 +74,31 @@ def test_cfg4_long_context_full_depth(weights_1p5b):
     cfg, ses, gpu, ref, stats = _run_full("cfg4_1p5b_long", weights_1p5b, sample=[1, 6])
     ses.close()
     assert stats["logit_err"] <= P.LOGIT_TOL
+
+
+def test_cfg5_7b_shape_full_batch_reduced_depth():
+    """The 7B-shaped escalation verifier with its whole batch of 32 steps, full width and vocabulary, at 3 of its 28
+    layers (drawing all 15 GB of its weights on the host takes minutes): every kernel runs in the launch shapes of
+    the full model, only the loop over layers is shorter."""
+    from workloads import scaled_config
+    cfg = scaled_config("cfg5_7b_b32", n_layers=3)
+    weights = model_weights(cfg.model, cfg.seed)
+    batch = make_batch(cfg)
+    sample = [2, 17, 31]
+    ses = P.build_session(cfg, weights, batch)
+    try:
+        ses.verify()
+        gpu = ses.results()
+        ref = P.oracle_outputs(cfg, weights, batch, steps=sample)
+        stats = P.compare(gpu, ses.last_logits(), ref, cfg.tau, steps=sample, gpu_lse=ses.last_lse())
+        P.check_verdict(gpu, ref, cfg.verdict_ids, steps=sample)
+        assert stats["logit_err"] <= P.LOGIT_TOL
+    finally:
+        ses.close()
+
+
+def test_cfg5_7b_shape_full_depth():
+    """All 28 layers of the 7B-shaped verifier (15 GB of weights), whole batch; the oracle recomputes two steps."""
+    _, ses, gpu, ref, stats = _run_full("cfg5_7b_b32", None, sample=[5, 28])
+    ses.close()
+    assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
