@@ -320,19 +320,27 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_slot;
-  // Set-up overlapped the previous kernel's tail; q, k, v of the new tokens are needed from here on.
+  // Set-up overlapped the previous kernel's tail; q, k, v of the new tokens are needed from here on. The producer
+  // warps wait a little later: the cached pages do not depend on the previous kernel, so they first send for the
+  // cached tiles that fit their rings.
   pdl_launch_dependents();
-  pdl_wait();
+  if (warp != 0 && warp != 6) pdl_wait();
 
   if (warp == 0 || warp == 6) {
     // ------------------------------------------------------------ TMA producers (whole warps): warp 0 K, warp 6 V
     const bool is_k = warp == 0;
-    if (is_k && lane == 0) {
-      mbar_arrive_expect_tx(&bars->q_full, L::kHalves * (128 / G) * G * 128);
+    bool waited = false;
+    auto dependency_wait = [&]() {
+      if (waited) return;
+      pdl_wait();
+      waited = true;
+      if (is_k && lane == 0) {
+        mbar_arrive_expect_tx(&bars->q_full, L::kHalves * (128 / G) * G * 128);
 #pragma unroll
-      for (int h = 0; h < L::kHalves; ++h)
-        tma_load_3d(smem + L::kQOff + h * 128 * 128, &tm_q3d, &bars->q_full, h * 64, it.kv_head * G, tok0 + it.q_tok0);
-    }
+        for (int h = 0; h < L::kHalves; ++h)
+          tma_load_3d(smem + L::kQOff + h * 128 * 128, &tm_q3d, &bars->q_full, h * 64, it.kv_head * G, tok0 + it.q_tok0);
+      }
+    };
     const int32_t* pages = p.page_table + static_cast<size_t>(it.seq) * p.max_pages_per_seq;
     const int n_pages = (ctx + kPage - 1) / kPage;
     // Lane l < 8 fetches page l of a cached tile. Pages past the end of the context are replaced by the last
@@ -351,6 +359,8 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
     uint32_t phase = 0;
     bool ok = true;
     for (int t = it.tile_begin; t < it.tile_end; ++t) {
+      // the first cached tiles, as many as the ring holds, go out before the previous kernel is known to be complete
+      if (t >= ctx_tiles || t - it.tile_begin >= kStages) dependency_wait();
       const int next_page = page_of(t + 1 < it.tile_end ? t + 1 : t);
       const int group = ((page * p.n_kv_heads + it.kv_head) * kPage) >> 3;     // 8-row group within a K or V plane
       uint8_t* dst = ring + stage * L::kTileBytes;
@@ -369,6 +379,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
       page = next_page;
       if (++stage == kStages) { stage = 0; phase ^= 1u; }
     }
+    dependency_wait();
     // In a healthy run the MMA warp has waited for every copy before the CTA exits. After an abort, give
     // the copies still in flight time to land in shared memory before the CTA may go away.
     if (!ok)

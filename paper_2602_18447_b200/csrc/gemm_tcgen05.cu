@@ -172,6 +172,20 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
   // Everything above overlapped the previous kernel's tail; its results (the A operand, x) are needed from here on.
   pdl_launch_dependents();
+  // The producer thread waits a little later: the weights do not depend on the previous kernel, so it first sends
+  // for the B boxes of its first stages (all stages are empty at this point).
+  const int pre = (threadIdx.x == 0) ? max(0, min(L::kStages, end - start)) : 0;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < pre; ++i) {
+      const int u = start + i, tile = u / kblocks, kb = u - tile * kblocks;
+      const int n0 = tile_n(tile, m_tiles, n_tiles, EPI) * OUT_BN;
+      uint8_t* sb = smem + i * L::kStageBytes + kABytes;
+      mbar_arrive_expect_tx(&full_bar[i], L::kStageBytes);
+      tma_load_2d(sb, &tm_b, &full_bar[i], kb * BK, n0);
+      if (EPI == kEpiSwiGLU) tma_load_2d(sb + 128 * BK * 2, &tm_b2, &full_bar[i], kb * BK, n0);
+      else if (BN == 256) tma_load_2d(sb + 128 * BK * 2, &tm_b, &full_bar[i], kb * BK, n0 + 128);
+    }
+  }
   pdl_wait();
 
   if (warp == 0) {
@@ -179,22 +193,27 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // One thread issues the two or three 16 KB boxes of a stage in turn. (Spreading them over lanes of the warp,
     // which pays for 4 KB boxes, was measured slower here.)
     if (lane == 0) {
-      int stage = 0;
+      int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int u = start; u < end && ok;) {
         const Segment sg = next_segment(u, end, kblocks);
         const int m0 = tile_m(sg.tile, m_tiles, n_tiles, EPI) * BM;
         const int n0 = tile_n(sg.tile, m_tiles, n_tiles, EPI) * OUT_BN;
-        for (int kb = sg.kb0; kb < sg.kb0 + sg.len; ++kb) {
-          if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
+        for (int kb = sg.kb0; kb < sg.kb0 + sg.len; ++kb, ++issued) {
           uint8_t* sa = smem + stage * L::kStageBytes;
           uint8_t* sb = sa + kABytes;
-          mbar_arrive_expect_tx(&full_bar[stage], L::kStageBytes);
-          tma_load_2d(sa, &tm_a, &full_bar[stage], kb * BK, m0);
-          tma_load_2d(sb, &tm_b, &full_bar[stage], kb * BK, n0);
-          if (EPI == kEpiSwiGLU) tma_load_2d(sb + 128 * BK * 2, &tm_b2, &full_bar[stage], kb * BK, n0);
-          else if (BN == 256) tma_load_2d(sb + 128 * BK * 2, &tm_b, &full_bar[stage], kb * BK, n0 + 128);
+          if (issued < pre) {
+            // first use of the stage: its bytes are announced and its weight boxes already on their way
+            tma_load_2d(sa, &tm_a, &full_bar[stage], kb * BK, m0);
+          } else {
+            if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
+            mbar_arrive_expect_tx(&full_bar[stage], L::kStageBytes);
+            tma_load_2d(sa, &tm_a, &full_bar[stage], kb * BK, m0);
+            tma_load_2d(sb, &tm_b, &full_bar[stage], kb * BK, n0);
+            if (EPI == kEpiSwiGLU) tma_load_2d(sb + 128 * BK * 2, &tm_b2, &full_bar[stage], kb * BK, n0);
+            else if (BN == 256) tma_load_2d(sb + 128 * BK * 2, &tm_b, &full_bar[stage], kb * BK, n0 + 128);
+          }
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
         u += sg.len;
