@@ -34,8 +34,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) of one gate/up GEMM launch of the default workload, from the ncu capture summarised in
 # profiles/gemm_f16_cfg2_4layers.md, and the hash of the kernel source that capture was taken with. A changed kernel
 # has no counters: traffic is then reported as null.
-GATEUP_TRAFFIC = {"workload": "cfg2_1p5b_b16", "bytes": 58.653696e6 + 4.392448e6,
-                  "source": "paper_2602_18447_b200/csrc/gemm_tcgen05.cu", "sha256_16": "af754d5552c638da"}
+GATEUP_TRAFFIC = {"workload": "cfg2_1p5b_b16", "bytes": 58.657792e6 + 4.34688e6,
+                  "source": "paper_2602_18447_b200/csrc/gemm_tcgen05.cu", "sha256_16": "25b6cee4a6e08f25"}
 
 
 def gateup_traffic(workload: str):
@@ -291,6 +291,7 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
     barrier()
     ms_e2e = e0.elapsed_time(e1)
+    h2d_bytes = B.cs_last_h2d_bytes(ses.model)     # tokens + batch metadata, one pinned block per call
 
     # ---- per-kernel durations (events around every launch; same workload, same process) -------------
     B.cs_profile(ses.model, True)
@@ -344,7 +345,7 @@ def run_ours(args, cfg):
                    "replicas": world},
         "clocks": clocks,
         "e2e": {"value": all_steps * K / (ms_e2e * 1e-3), "unit": UNIT,
-                "h2d_bytes_per_step": int(batch.n_tokens * 4 + (6 * batch.n_steps + 2 * batch.n_tokens) * 4),
+                "h2d_bytes_per_step": int(h2d_bytes),
                 "d2h_bytes_per_step": int(batch.n_steps * 5), "ms_per_step": ms_e2e / K},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "gemm_f16_kernel<256, SwiGLU> (gate/up projection)", "bound": "tensor",

@@ -278,6 +278,9 @@ int cs_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d
 #define CS_PROF_CLASSES 11
 int cs_profile(cs_model* model, int enable);
 int cs_profile_read(cs_model* model, float* ms_out, int32_t* calls_out, int n_classes);
+/* Bytes that the last cs_verify_steps / cs_prefill call on this model copied from the host to the device: the batch
+ * metadata (offsets, positions, attention work items) and, when the tokens were given on the host, the tokens. */
+int64_t cs_last_h2d_bytes(const cs_model* model);
 /* Number of kernels the library has launched on this host thread since the last call of this function. */
 int64_t cs_take_launch_count(void);
 

@@ -17,7 +17,7 @@ EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_reserve",
     "cs_kv_alloc", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
     "cs_verify_steps", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
-    "cs_last_status", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_profile", "cs_profile_read",
+    "cs_last_status", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
 ]
 
 PROF_CLASSES = ["embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gateup", "gemm_down",
@@ -84,6 +84,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_lm_head_gate": (C.c_int, [vp, vp, i32, i32, i32, vp, i32, f32, vp, vp, vp, vp, vp]),
         "cs_lm_head_gate_static": (C.c_int, [vp, vp, i32, i32, i32, vp, i32, f32, vp, vp, vp, vp, vp]),
         "cs_take_launch_count": (C.c_int64, []),
+        "cs_last_h2d_bytes": (C.c_int64, [vp]),
         "cs_profile": (C.c_int, [vp, i32]),
         "cs_profile_read": (C.c_int, [vp, vp, vp, i32]),
     }
@@ -133,6 +134,10 @@ def _stream_ptr(stream) -> Optional[int]:
 
 def cs_version() -> int:
     return load_library().cs_version()
+
+
+def cs_last_h2d_bytes(model: int) -> int:
+    return int(load_library().cs_last_h2d_bytes(model))
 
 
 def cs_take_launch_count() -> int:

@@ -99,6 +99,7 @@ struct cs_model {
   Staging stg;
   bool keep_logits = false;
   int last_B = 0;
+  int64_t last_h2d_bytes = 0;   // bytes the last cs_verify_steps / cs_prefill call copied to the device
   Prof prof;
 };
 
@@ -457,6 +458,7 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   }
   if (!items.empty()) std::memcpy(h + L.off_items, items.data(), items.size() * sizeof(AttnItem));
   CS_CUDA(cudaMemcpyAsync(m->stg.dev.p, h, L.total * 4, cudaMemcpyHostToDevice, s));
+  m->last_h2d_bytes = static_cast<int64_t>(L.total) * 4;
   CS_CUDA(cudaEventRecord(m->stg.ev[slot], s));
   m->stg.pending[slot] = true;
   *out = L;
@@ -815,6 +817,8 @@ int cs_cascade_select(const uint8_t* trusted, const int32_t* verdict_d, const fl
                                 out_prefix_len, out_best, out_pass, out_conf, static_cast<cudaStream_t>(stream)));
   return CS_OK;
 }
+
+int64_t cs_last_h2d_bytes(const cs_model* m) { return m ? m->last_h2d_bytes : 0; }
 
 int cs_set_keep_logits(cs_model* m, int keep) {
   if (!m) return CS_EINVAL;
