@@ -272,8 +272,9 @@ int cs_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d
  * of CUDA events around each kernel launch (on the call's stream); cs_profile_read waits for the recorded
  * events, adds the elapsed milliseconds and the number of timed launches per class into ms_out / calls_out
  * (host arrays of n_classes >= CS_PROF_CLASSES entries) and clears the record. Classes, in order: embedding,
- * RMSNorm, QKV GEMM, rotary, attention (+ merge), O GEMM, gate/up GEMM (SwiGLU), down GEMM, LM head, gate,
- * other. The events cost a little host and device time, so throughput is measured with profiling off.
+ * RMSNorm, QKV GEMM (rotary turn in its epilogue), rotary (unused: always 0), attention, O GEMM, gate/up GEMM (SwiGLU),
+ * down GEMM, LM head, gate, other. The events keep consecutive kernels from overlapping and cost a little host and
+ * device time, so throughput is measured with profiling off.
  */
 #define CS_PROF_CLASSES 11
 int cs_profile(cs_model* model, int enable);
