@@ -25,7 +25,9 @@ shift invariance, GQA == MHA with repeated heads, softmax sums to one, gate
 end points of Table 3 (gamma = 0 never escalates, gamma > 1 always does),
 batch-permutation equivariance, the whole forward against the
 `transformers` Qwen2 architecture used as a black-box library routine, and hand-worked iterations of
-Algorithm 1 / Eq. 5 for the selection bookkeeping (tests/golden/cascade_cases.txt).
+Algorithm 1 / Eq. 5 for the selection bookkeeping (tests/golden/cascade_cases.txt); for the two-tier
+verifier, its reduction to one tier at either end of the threshold and the rule of Eq. 4 applied step by step
+to two independent full-batch runs (tests/test_oracle_cascade.py).
 """
 from __future__ import annotations
 
@@ -280,3 +282,32 @@ def verify_steps(weights: dict, tokens_per_step: List[np.ndarray], ctx_lens: Seq
     logits = last_position_logits(weights, xs)
     conf, verdict, lse = verdict_confidence(logits, verdict_ids)
     return {"logits": logits, "conf": conf, "verdict": verdict, "lse": lse, "accept": gate(conf, tau)}
+
+
+def verify_cascade(weights_d: dict, weights_t: dict, tokens_per_step: List[np.ndarray],
+                   ctx_lens: Sequence[int], ctx_kv_fn_d, ctx_kv_fn_t,
+                   verdict_ids: Sequence[int], tau: float) -> dict:
+    """The two-tier verifier V_cascade (Eq. 4; Algorithm 1, Stage 2): every step goes through the draft
+    model; the steps whose draft confidence is below gamma, and only those, go through the target model;
+    the final decision of a step is r_D where p_D >= gamma and r_T otherwise.
+
+    ctx_kv_fn_d / ctx_kv_fn_t (step, layer) -> (K, V): the same reasoning context as cached by each model,
+    indexed by the step's position in the full batch.
+    Returns the draft tier's dict under "draft", the target tier's under "target" (its arrays run over the
+    escalated steps only, in ascending step order; None when nothing was escalated), "escalated" (their
+    step indices), and per step of the batch "verdict" (final decision) and "conf" (confidence of the
+    verifier whose decision was taken)."""
+    draft = verify_steps(weights_d, tokens_per_step, ctx_lens, ctx_kv_fn_d, verdict_ids, tau)
+    escalated = [i for i in range(len(tokens_per_step)) if not draft["accept"][i]]
+    verdict = np.array(draft["verdict"], dtype=np.int32)
+    conf = np.array(draft["conf"], dtype=np.float64)
+    target = None
+    if escalated:
+        target = verify_steps(weights_t, [tokens_per_step[i] for i in escalated],
+                              [ctx_lens[i] for i in escalated],
+                              lambda j, l: ctx_kv_fn_t(escalated[j], l), verdict_ids, tau)
+        for j, i in enumerate(escalated):
+            verdict[i] = target["verdict"][j]
+            conf[i] = target["conf"][j]
+    return {"draft": draft, "target": target, "escalated": np.array(escalated, dtype=np.int32),
+            "verdict": verdict, "conf": conf}
