@@ -180,6 +180,36 @@ int cs_escalate_mask(const float* conf, int B, float tau, uint8_t* out_accept,
                      int32_t* out_escalate_idx, int32_t* out_escalate_count, void* stream);
 
 /*
+ * cs_verify_cascade - the two-tier verifier V_cascade of Eq. 4 (Algorithm 1, Stage 2) in one call: every step goes
+ * through the draft model (cs_verify_steps); the steps whose confidence p_D is below gamma are listed on the device
+ * (cs_escalate_mask) and go, as one smaller batch, through the target model; the final decision of a step is r_D
+ * where p_D >= gamma and r_T otherwise. The target model therefore costs time in proportion to the cascade rate
+ * (Section 4.4).
+ *   draft, kv_d        draft model and its context cache; target, kv_t likewise (draft != target). Sequence
+ *                      seq_ids[i] must be set in BOTH caches and hold the same reasoning context as each model
+ *                      caches it. The models may differ in every dimension; token and verdict ids must be valid in both.
+ *   seq_ids, step_lens host int32[B];  step_tokens  HOST int32[sum step_lens] (the second batch is laid out on
+ *                      the host from the list of escalated steps).
+ *   out_conf_d, out_trusted, out_verdict_d   device float[B], uint8[B], int32[B]: the draft tier's p_D,
+ *                      (p_D >= tau), r_D as an index into verdict_ids. All required.
+ *   out_conf_t, out_verdict_t   device float[B], int32[B] or NULL: the target tier's p_T and r_T at the escalated
+ *                      steps, (0, -1) at the trusted ones.
+ *   out_verdict, out_conf   device int32[B], float[B]: final decision and the confidence of the verifier that
+ *                      took it. Required.
+ *   host_n_escalated   host int32[1] or NULL: number of escalated steps, valid on return.
+ * The call blocks the host once between the tiers (it reads the list back: 4 (B + 1) bytes); the target pass and
+ * the final scatter are asynchronous on `stream`. Arguments are checked for both tiers before anything is
+ * launched. B <= 65536.
+ * Errors: as cs_verify_steps.
+ */
+int cs_verify_cascade(cs_model* draft, const cs_kv* kv_d, cs_model* target, const cs_kv* kv_t,
+                      const int32_t* seq_ids, int B, const int32_t* step_tokens, const int32_t* step_lens,
+                      const int32_t* verdict_ids, int n_verdict, float tau,
+                      float* out_conf_d, uint8_t* out_trusted, int32_t* out_verdict_d,
+                      float* out_conf_t, int32_t* out_verdict_t, int32_t* out_verdict, float* out_conf,
+                      int32_t* host_n_escalated, void* stream);
+
+/*
  * cs_cascade_select - what the drafting loop does with the verification results of one iteration, on the device.
  * Final decision of step i (Algorithm 1, Stage 2; Eq. 4): the draft verifier's decision when it was trusted
  * (trusted[i] != 0, i.e. p_D >= gamma), else the target verifier's; an escalated step without a target result

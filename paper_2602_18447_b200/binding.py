@@ -16,7 +16,7 @@ CS_OK, CS_EINVAL, CS_ENOMEM, CS_ECUDA, CS_ETIMEOUT, CS_ESTATE, CS_ELIMIT = range
 EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_reserve",
     "cs_kv_alloc", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
-    "cs_verify_steps", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
+    "cs_verify_steps", "cs_verify_cascade", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
     "cs_last_status", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
 ]
 
@@ -73,6 +73,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_kv_fill": (C.c_int, [vp, i32, i32, vp, vp, vp]),
         "cs_prefill": (C.c_int, [vp, vp, vp, vp, vp, i32, vp]),
         "cs_verify_steps": (C.c_int, [vp, vp, vp, i32, vp, i32, vp, vp, i32, f32, vp, vp, vp, vp]),
+        "cs_verify_cascade": (C.c_int, [vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
         "cs_escalate_mask": (C.c_int, [vp, i32, f32, vp, vp, vp, vp]),
         "cs_cascade_select": (C.c_int, [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]),
         "cs_set_keep_logits": (C.c_int, [vp, i32]),
@@ -231,6 +232,28 @@ def cs_verify_steps(model: int, ctx_kv: int, seq_ids, step_tokens, step_lens, ve
                                           _np_ptr(v), int(v.shape[0]), float(tau), _dev_ptr(out_conf),
                                           _dev_ptr(out_accept), _dev_ptr(out_verdict), _stream_ptr(stream)),
            "cs_verify_steps")
+
+
+def cs_verify_cascade(draft: int, kv_d: int, target: int, kv_t: int, seq_ids, step_tokens, step_lens,
+                      verdict_ids: Sequence[int], tau: float, out_conf_d, out_trusted, out_verdict_d, out_conf_t,
+                      out_verdict_t, out_verdict, out_conf, stream=None) -> int:
+    """step_tokens: host int32 (numpy or a CPU torch tensor). The out_* are CUDA tensors of length B (out_conf_t and
+    out_verdict_t may be None). Returns the number of escalated steps."""
+    s, l, v = _i32(seq_ids), _i32(step_lens), _i32(verdict_ids)
+    if hasattr(step_tokens, "is_cuda"):
+        if step_tokens.is_cuda:
+            raise ValueError("cs_verify_cascade takes the step tokens in host memory")
+        tok_ptr = step_tokens.data_ptr()
+    else:
+        step_tokens = _i32(step_tokens)
+        tok_ptr = _np_ptr(step_tokens)
+    n_esc = C.c_int32(0)
+    _check(load_library().cs_verify_cascade(draft, kv_d, target, kv_t, _np_ptr(s), int(s.shape[0]), tok_ptr, _np_ptr(l),
+                                            _np_ptr(v), int(v.shape[0]), float(tau), _dev_ptr(out_conf_d),
+                                            _dev_ptr(out_trusted), _dev_ptr(out_verdict_d), _dev_ptr(out_conf_t),
+                                            _dev_ptr(out_verdict_t), _dev_ptr(out_verdict), _dev_ptr(out_conf),
+                                            C.cast(C.byref(n_esc), C.c_void_p), _stream_ptr(stream)), "cs_verify_cascade")
+    return int(n_esc.value)
 
 
 def cs_escalate_mask(conf, tau: float, out_accept, out_escalate_idx, out_escalate_count, stream=None) -> None:

@@ -100,6 +100,10 @@ struct cs_model {
   bool keep_logits = false;
   int last_B = 0;
   int64_t last_h2d_bytes = 0;   // bytes the last cs_verify_steps / cs_prefill call copied to the device
+  // two-tier pass: list of escalated steps (+ its length) on the draft model, compact results on the target model
+  DevBuf casc_idx, casc_conf, casc_verdict, casc_accept;
+  int32_t* casc_host = nullptr;   // pinned copy of the list
+  size_t casc_host_cap = 0;
   Prof prof;
 };
 
@@ -603,8 +607,10 @@ int cs_model_free(cs_model* m) {
   cudaDeviceSynchronize();
   for (void* p : m->owned) cudaFree(p);
   DevBuf* bufs[] = {&m->x, &m->a, &m->qkv, &m->attn_o, &m->hmlp, &m->rope, &m->h_last, &m->lm_part, &m->vlogits,
-                    &m->logits, &m->lse, &m->attn_part_o, &m->attn_part_ml, &m->attn_counters, &m->stg.dev};
+                    &m->logits, &m->lse, &m->attn_part_o, &m->attn_part_ml, &m->attn_counters, &m->stg.dev,
+                    &m->casc_idx, &m->casc_conf, &m->casc_verdict, &m->casc_accept};
   for (DevBuf* b : bufs) b->release();
+  if (m->casc_host) cudaFreeHost(m->casc_host);
   for (cudaEvent_t e : m->prof.pool) cudaEventDestroy(e);
   for (int i = 0; i < kStagingRing; ++i) {
     if (m->stg.host[i]) cudaFreeHost(m->stg.host[i]);
@@ -803,6 +809,89 @@ int cs_escalate_mask(const float* conf, int B, float tau, uint8_t* out_accept, i
   if (B < 0 || B > 65536 || tau != tau || !out_count) return CS_EINVAL;
   if (B > 0 && (!conf || !out_idx)) return CS_EINVAL;
   CS_CUDA(launch_escalate(conf, B, tau, out_accept, out_idx, out_count, static_cast<cudaStream_t>(stream)));
+  return CS_OK;
+}
+
+int cs_verify_cascade(cs_model* draft, const cs_kv* kv_d, cs_model* target, const cs_kv* kv_t, const int32_t* seq_ids,
+                      int B, const int32_t* step_tokens, const int32_t* step_lens, const int32_t* verdict_ids,
+                      int n_verdict, float tau, float* out_conf_d, uint8_t* out_trusted, int32_t* out_verdict_d,
+                      float* out_conf_t, int32_t* out_verdict_t, int32_t* out_verdict, float* out_conf,
+                      int32_t* host_n_escalated, void* stream) {
+  if (!draft || !target || draft == target || !kv_d || !kv_t || kv_d->model != draft || kv_t->model != target || B < 0)
+    return CS_EINVAL;
+  if (tau != tau || n_verdict < 1 || n_verdict > 8 || !verdict_ids) return CS_EINVAL;
+  for (int j = 0; j < n_verdict; ++j)
+    if (verdict_ids[j] < 0 || verdict_ids[j] >= draft->d.vocab || verdict_ids[j] >= target->d.vocab) return CS_EINVAL;
+  if (host_n_escalated) *host_n_escalated = 0;
+  if (B == 0) return CS_OK;
+  if (B > 65536) return CS_EINVAL;
+  if (!seq_ids || !step_tokens || !step_lens || !out_conf_d || !out_trusted || !out_verdict_d || !out_verdict ||
+      !out_conf)
+    return CS_EINVAL;
+  // everything the target pass would reject is rejected before the draft pass is launched
+  {
+    int64_t t = 0;
+    for (int i = 0; i < B; ++i) {
+      if (step_lens[i] < 1 || seq_ids[i] < 0 || seq_ids[i] >= kv_t->max_seqs || seq_ids[i] >= kv_d->max_seqs)
+        return CS_EINVAL;
+      if (kv_t->ctx_len[seq_ids[i]] < 0 || kv_d->ctx_len[seq_ids[i]] < 0) return CS_ESTATE;
+      t += step_lens[i];
+    }
+    for (int64_t k = 0; k < t; ++k)
+      if (step_tokens[k] < 0 || step_tokens[k] >= target->d.vocab) return CS_EINVAL;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc;
+  if ((rc = draft->casc_idx.ensure(sizeof(int32_t) * (static_cast<size_t>(B) + 1)))) return rc;
+  if (draft->casc_host_cap < static_cast<size_t>(B) + 1) {
+    if (draft->casc_host) cudaFreeHost(draft->casc_host);
+    draft->casc_host = nullptr;
+    draft->casc_host_cap = 0;
+    const size_t want = 2 * static_cast<size_t>(B) + 64;
+    CS_CUDA(cudaMallocHost(reinterpret_cast<void**>(&draft->casc_host), want * sizeof(int32_t)));
+    draft->casc_host_cap = want;
+  }
+  // tier 1: every step through the draft model
+  if ((rc = cs_verify_steps(draft, kv_d, seq_ids, B, step_tokens, 0, step_lens, verdict_ids, n_verdict, tau, out_conf_d,
+                            out_trusted, out_verdict_d, stream)))
+    return rc;
+  // the steps it is not confident about, listed on the device; the host needs the list to lay out the second batch
+  int32_t* idx = static_cast<int32_t*>(draft->casc_idx.p);
+  int32_t* count = idx + B;
+  CS_CUDA(launch_escalate(out_conf_d, B, tau, nullptr, idx, count, s));
+  CS_CUDA(cudaMemcpyAsync(draft->casc_host + B, count, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  CS_CUDA(cudaMemcpyAsync(draft->casc_host, idx, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
+  CS_CUDA(cudaStreamSynchronize(s));
+  const int n_esc = draft->casc_host[B];
+  if (n_esc < 0 || n_esc > B) return CS_ECUDA;
+  if (host_n_escalated) *host_n_escalated = n_esc;
+  // tier 2: the escalated steps, as one smaller batch, through the target model
+  const int32_t* verdict_c = nullptr;
+  const float* conf_c = nullptr;
+  if (n_esc > 0) {
+    if ((rc = target->casc_conf.ensure(sizeof(float) * n_esc))) return rc;
+    if ((rc = target->casc_verdict.ensure(sizeof(int32_t) * n_esc))) return rc;
+    if ((rc = target->casc_accept.ensure(n_esc))) return rc;
+    std::vector<int64_t> cu(static_cast<size_t>(B) + 1, 0);
+    for (int i = 0; i < B; ++i) cu[i + 1] = cu[i] + step_lens[i];
+    std::vector<int32_t> sub_seq(n_esc), sub_len(n_esc), sub_tok;
+    for (int j = 0; j < n_esc; ++j) {
+      const int i = draft->casc_host[j];
+      if (i < 0 || i >= B) return CS_ECUDA;
+      sub_seq[j] = seq_ids[i];
+      sub_len[j] = step_lens[i];
+      sub_tok.insert(sub_tok.end(), step_tokens + cu[i], step_tokens + cu[i + 1]);
+    }
+    if ((rc = cs_verify_steps(target, kv_t, sub_seq.data(), n_esc, sub_tok.data(), 0, sub_len.data(), verdict_ids,
+                              n_verdict, tau, static_cast<float*>(target->casc_conf.p),
+                              static_cast<uint8_t*>(target->casc_accept.p),
+                              static_cast<int32_t*>(target->casc_verdict.p), stream)))
+      return rc;
+    verdict_c = static_cast<const int32_t*>(target->casc_verdict.p);
+    conf_c = static_cast<const float*>(target->casc_conf.p);
+  }
+  CS_CUDA(launch_cascade_scatter(B, out_trusted, out_verdict_d, out_conf_d, idx, count, verdict_c, conf_c, out_verdict_t,
+                                 out_conf_t, out_verdict, out_conf, s));
   return CS_OK;
 }
 

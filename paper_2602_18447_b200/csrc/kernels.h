@@ -92,6 +92,12 @@ cudaError_t launch_cascade_select(const uint8_t* trusted, const int32_t* verdict
                                   float* out_conf, cudaStream_t s);
 cudaError_t launch_escalate(const float* conf, int B, float tau, uint8_t* out_accept, int32_t* out_idx,
                             int32_t* out_count, cudaStream_t s);
+// Results of the target pass (compact, over the escalated steps idx[0 .. *count)) back to batch order, and the
+// final decision of Eq. 4 for every step.
+cudaError_t launch_cascade_scatter(int B, const uint8_t* trusted, const int32_t* verdict_d, const float* conf_d,
+                                   const int32_t* idx, const int32_t* count, const int32_t* verdict_c,
+                                   const float* conf_c, int32_t* out_verdict_t, float* out_conf_t,
+                                   int32_t* out_verdict, float* out_conf, cudaStream_t s);
 
 // Launch with programmatic stream serialisation (see pdl_wait in common.cuh).
 template <typename... KArgs, typename... Args>

@@ -322,6 +322,39 @@ __global__ void escalate_kernel(const float* __restrict__ conf, int B, float tau
   if (threadIdx.x == 0) *out_count = base;
 }
 
+// Eq. 4 per step, after the target pass over the escalated steps only: idx[0 .. *count) lists those steps in
+// ascending order and verdict_c / conf_c hold the target's results in that order. A trusted step keeps the draft's
+// decision and gets (-1, 0) as its target result; an escalated one takes the target's.
+__global__ void cascade_scatter_kernel(int B, const uint8_t* __restrict__ trusted, const int32_t* __restrict__ verdict_d,
+                                       const float* __restrict__ conf_d, const int32_t* __restrict__ idx,
+                                       const int32_t* __restrict__ count, const int32_t* __restrict__ verdict_c,
+                                       const float* __restrict__ conf_c, int32_t* __restrict__ out_verdict_t,
+                                       float* __restrict__ out_conf_t, int32_t* __restrict__ out_verdict,
+                                       float* __restrict__ out_conf) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B) return;
+  int v = verdict_d[i], vt = -1;
+  float c = conf_d[i], ct = 0.f;
+  if (!trusted[i]) {
+    const int n = *count;
+    int lo = 0, hi = n;                 // position of i in the ascending list
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (idx[mid] < i) lo = mid + 1; else hi = mid;
+    }
+    if (lo < n && idx[lo] == i) {
+      vt = verdict_c[lo];
+      ct = conf_c[lo];
+    }
+    v = vt;
+    c = ct;
+  }
+  if (out_verdict_t) out_verdict_t[i] = vt;
+  if (out_conf_t) out_conf_t[i] = ct;
+  out_verdict[i] = v;
+  out_conf[i] = c;
+}
+
 // One warp per request: final decision and confidence of each of its steps (Eq. 4), the length of the leading run
 // of accepted steps (Algorithm 1's loop with break) and the accepted step with the highest confidence (Eq. 5).
 __global__ void cascade_select_kernel(const uint8_t* __restrict__ trusted, const int32_t* __restrict__ verdict_d,
@@ -454,6 +487,17 @@ cudaError_t launch_cascade_select(const uint8_t* trusted, const int32_t* verdict
   cascade_select_kernel<<<(R + warps - 1) / warps, warps * 32, 0, s>>>(trusted, verdict_d, conf_d, verdict_t, conf_t,
                                                                      req_offsets, R, accept_index, out_prefix_len,
                                                                      out_best, out_pass, out_conf);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_cascade_scatter(int B, const uint8_t* trusted, const int32_t* verdict_d, const float* conf_d,
+                                   const int32_t* idx, const int32_t* count, const int32_t* verdict_c,
+                                   const float* conf_c, int32_t* out_verdict_t, float* out_conf_t,
+                                   int32_t* out_verdict, float* out_conf, cudaStream_t s) {
+  if (B <= 0) return cudaSuccess;
+  cascade_scatter_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, trusted, verdict_d, conf_d, idx, count, verdict_c, conf_c,
+                                                         out_verdict_t, out_conf_t, out_verdict, out_conf);
   count_launch();
   return cudaGetLastError();
 }

@@ -99,3 +99,39 @@ class VerifySession:
 
     def __exit__(self, *exc):
         self.close()
+
+
+class CascadeSession:
+    """A draft and a target VerifySession over the same batch (each model caches the same contexts under the same
+    sequence ids) and the outputs of the two-tier pass."""
+
+    def __init__(self, draft: VerifySession, target: VerifySession):
+        assert draft.n_steps == target.n_steps
+        self.draft, self.target = draft, target
+        n, dev = draft.n_steps, draft.device
+        self.out_conf_t = torch.empty(n, dtype=torch.float32, device=dev)
+        self.out_verdict_t = torch.empty(n, dtype=torch.int32, device=dev)
+        self.out_conf = torch.empty(n, dtype=torch.float32, device=dev)
+        self.out_verdict = torch.empty(n, dtype=torch.int32, device=dev)
+        self.n_escalated = -1
+
+    def verify(self, tau: Optional[float] = None, stream=None) -> int:
+        d = self.draft
+        self.n_escalated = B.cs_verify_cascade(
+            d.model, d.kv, self.target.model, self.target.kv, d.seq_ids, d.tokens_pinned, d.batch.step_lens,
+            d.cfg.verdict_ids, d.cfg.tau if tau is None else tau, d.out_conf, d.out_accept, d.out_verdict,
+            self.out_conf_t, self.out_verdict_t, self.out_verdict, self.out_conf, stream=stream)
+        return self.n_escalated
+
+    def results(self) -> dict:
+        torch.cuda.synchronize()
+        B.cs_last_status(self.draft.model)
+        B.cs_last_status(self.target.model)
+        return {"conf_d": self.draft.out_conf.cpu().numpy(), "trusted": self.draft.out_accept.cpu().numpy(),
+                "verdict_d": self.draft.out_verdict.cpu().numpy(), "conf_t": self.out_conf_t.cpu().numpy(),
+                "verdict_t": self.out_verdict_t.cpu().numpy(), "conf": self.out_conf.cpu().numpy(),
+                "verdict": self.out_verdict.cpu().numpy(), "n_escalated": self.n_escalated}
+
+    def close(self) -> None:
+        self.draft.close()
+        self.target.close()

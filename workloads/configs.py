@@ -85,6 +85,41 @@ CONFIGS = {
 }
 
 
+@dataclass(frozen=True)
+class CascadeConfig:
+    """Two-tier verification (Eq. 4): the batch recipe, threshold and draft verifier of `draft`, plus the shape
+    and weight seed of the target verifier that re-verifies the escalated steps. Both models cache the same
+    contexts; the batch (token ids, lengths) is the draft config's."""
+    name: str
+    draft: VerifyConfig
+    target_model: ModelShape
+    target_seed: int
+
+    @property
+    def target(self) -> VerifyConfig:
+        """The draft's recipe with the target's shape and seed: for drawing the target's weights and its cached
+        context K/V. Its batch is NOT drawn from this (the seeds differ); both tiers share the draft's batch."""
+        return replace(self.draft, name=self.name + "_target", model=self.target_model, seed=self.target_seed)
+
+
+TINY_TARGET = ModelShape("tiny-target", 3, 384, 6, 2, 64, 1024, 4096, 1.0e4)
+
+CASCADES = {
+    "cascade_tiny": CascadeConfig(
+        "cascade_tiny", replace(CONFIGS["cfg1_tiny"], batch=12), TINY_TARGET, 111),
+    "cascade_1p5b_7b": CascadeConfig(
+        "cascade_1p5b_7b", CONFIGS["cfg2_1p5b_b16"], QWEN_7B, 606),
+}
+
+
+def get_cascade(name: str, *, target_layers: int | None = None) -> CascadeConfig:
+    c = CASCADES[name]
+    if target_layers is not None:
+        tm = replace(c.target_model, n_layers=target_layers, name=f"{c.target_model.name}-L{target_layers}")
+        c = replace(c, target_model=tm)
+    return c
+
+
 def get_config(name: str) -> VerifyConfig:
     return CONFIGS[name]
 
