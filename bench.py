@@ -2,6 +2,7 @@
 """Throughput of the batched draft-verification pass.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+    python bench.py --cascade cascade_1p5b_7b [--steps K] [--warmup W]     (two-tier pass, one GPU; see run_cascade)
 
 One "step" is one cs_verify_steps call over the whole batch of the workload (every kernel of the pass).
 Prints ONE JSON line. With --gpus N > 1 (launched by torch.distributed.run) every rank runs an independent
@@ -23,7 +24,8 @@ sys.path.insert(0, ROOT)
 
 import numpy as np  # noqa: E402
 
-from workloads import context_kv, get_config, make_batch, model_weights, page_assignment, scaled_config  # noqa: E402
+from workloads import (context_kv, get_cascade, get_config, make_batch, model_weights, page_assignment,  # noqa: E402
+                       plant_verdict_rows, scaled_config)
 
 METRIC = "verified_steps_per_s"
 UNIT = "steps/s"
@@ -369,6 +371,94 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_cascade(args):
+    """Times cs_verify_cascade (draft pass, list of escalated steps, target pass over those steps, final decision)
+    on one GPU, host tokens in and the blocking read-back of the list inside the timed region, next to its two
+    tiers timed alone: the cost model of Section 4.4 predicts t(draft) + t(target on the escalated steps).
+    Both models get the planted verdict rows, otherwise every confidence is ~1/V and every step is escalated."""
+    import torch
+    from paper_2602_18447_b200 import VerifySession, binding as B
+    from paper_2602_18447_b200.runner import CascadeSession
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the pass has no CPU path")
+    torch.cuda.set_device(0)
+    casc = get_cascade(args.cascade, target_layers=args.layers)
+    batch = make_batch(casc.draft)
+    tiers = []
+    for cfg in (casc.draft, casc.target):
+        w = model_weights(cfg.model, cfg.seed)
+        plant_verdict_rows(w, cfg.verdict_ids, beta=float(np.log(cfg.model.vocab) + 0.5), seed=cfg.seed)
+        ses = VerifySession(cfg, w, batch)
+        del w
+        total, pages = page_assignment(cfg, batch.ctx_lens)
+        if cfg.ctx_kv == "prefill":
+            ses.alloc_cache(pages, total, batch.ctx_lens, room_for_prefill=True)
+            ses.prefill_context(batch.ctx_tokens)
+        else:
+            ses.alloc_cache(pages, total, batch.ctx_lens)
+            ses.fill_synthetic_context(lambda i, l, cfg=cfg: context_kv(cfg, i, l, int(batch.ctx_lens[i])))
+        B.cs_reserve(ses.model, batch.n_steps, batch.n_tokens)
+        tiers.append(ses)
+    cs = CascadeSession(*tiers)
+    tau = casc.draft.tau if args.tau is None else args.tau
+    stream = torch.cuda.current_stream()
+    K, W = args.steps, max(3, args.warmup)
+
+    def timed(fn):
+        for _ in range(W):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(K):
+            fn()
+            stream.synchronize()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / K
+
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(0).uuid).replace("GPU-", ""))
+    sampler.start()
+    B.cs_take_launch_count()
+    t0 = time.time()
+    ms = timed(lambda: cs.verify(tau=tau))
+    t1 = time.time()
+    launches = B.cs_take_launch_count() // (K + W)
+    n_esc = cs.n_escalated
+    res = cs.results()
+    ms_draft = timed(lambda: cs.draft.verify(tau=tau, host_tokens=True))
+    ms_target_all = timed(lambda: cs.target.verify(tau=tau, host_tokens=True))
+    # the target alone on exactly the escalated steps
+    esc = np.nonzero(res["trusted"] == 0)[0]
+    ms_target_esc = 0.0
+    if esc.size:
+        toks = np.concatenate([batch.step_tokens[batch.cu_new[i]:batch.cu_new[i + 1]] for i in esc]).astype(np.int32)
+        lens = batch.step_lens[esc].astype(np.int32)
+        oc = torch.empty(esc.size, dtype=torch.float32, device="cuda")
+        oa = torch.empty(esc.size, dtype=torch.uint8, device="cuda")
+        t = cs.target
+        ms_target_esc = timed(lambda: B.cs_verify_steps(t.model, t.kv, esc.astype(np.int32), toks, lens,
+                                                        casc.draft.verdict_ids, tau, oc, oa, None))
+    sampler.stop()
+    out = {
+        "metric": METRIC, "value": batch.n_steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+        "data": "synthetic",
+        "config": {"workload": casc.name, "draft": casc.draft.model.name, "target": casc.target.model.name,
+                   "batch": batch.n_steps, "new_tokens": int(batch.n_tokens), "ctx_tokens": int(batch.ctx_lens.sum()),
+                   "tau": tau, "n_escalated": int(n_esc), "cascade_rate": n_esc / batch.n_steps,
+                   "timing": "host tokens in, list of escalated steps read back between the tiers, host waits for "
+                             "the final decisions every step",
+                   "l2": "inputs larger than L2 (both models' weights streamed every step)"},
+        "tiers_ms": {"cascade": ms, "draft_alone": ms_draft, "target_alone_all_steps": ms_target_all,
+                     "target_alone_escalated_steps": ms_target_esc,
+                     "draft_plus_target_escalated": ms_draft + ms_target_esc},
+        "gpu_launches": int(launches), "clocks": sampler.summary(t0, t1),
+    }
+    cs.close()
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -380,7 +470,14 @@ def main():
     ap.add_argument("--layers", type=int, default=None,
                     help="run a reduced-depth copy of the workload (for profiler captures of single kernels); "
                          "not a benchmark configuration")
+    ap.add_argument("--cascade", default=None,
+                    help="time the two-tier pass of this cascade workload instead (one GPU; with --layers the target "
+                         "model runs at that depth)")
+    ap.add_argument("--tau", type=float, default=None, help="threshold of the two-tier pass (default: the workload's)")
     args = ap.parse_args()
+    if args.cascade is not None:
+        run_cascade(args)
+        return
     cfg = get_config(args.workload)
     if args.layers is not None:
         cfg = scaled_config(args.workload, n_layers=args.layers)
