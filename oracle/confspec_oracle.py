@@ -27,7 +27,8 @@ batch-permutation equivariance, the whole forward against the
 `transformers` Qwen2 architecture used as a black-box library routine, and hand-worked iterations of
 Algorithm 1 / Eq. 5 for the selection bookkeeping (tests/golden/cascade_cases.txt); for the two-tier
 verifier, its reduction to one tier at either end of the threshold and the rule of Eq. 4 applied step by step
-to two independent full-batch runs (tests/test_oracle_cascade.py).
+to two independent full-batch runs; for the append of accepted steps (Stage 3), its equality with a prefill
+of the concatenated tokens from an empty cache (tests/test_oracle_cascade.py).
 """
 from __future__ import annotations
 
@@ -311,3 +312,29 @@ def verify_cascade(weights_d: dict, weights_t: dict, tokens_per_step: List[np.nd
             conf[i] = target["conf"][j]
     return {"draft": draft, "target": target, "escalated": np.array(escalated, dtype=np.int32),
             "verdict": verdict, "conf": conf}
+
+
+def append_accepted_steps(weights: dict, ctx_kv: list, m: Sequence[int], req_offsets: Sequence[int],
+                          draft_steps: List[np.ndarray], store_bf16: bool) -> list:
+    """Context management of Algorithm 1, Stage 3: context <- context (+) s^_1 (+) ... (+) s^_m for every request
+    with m > 0, in terms of the cache. ctx_kv[r][layer] = (K, V) of request r's context; draft_steps[i] holds the
+    token ids of drafted step i (the candidates of request r are steps req_offsets[r] .. req_offsets[r+1]-1).
+    The accepted tokens run through the model on top of the cached context, and their K/V (rounded to bf16
+    values when `store_bf16`, the cache format) are appended; requests with m = 0 keep their context as it is
+    (their next step comes from the target model's generation, which is outside this pass).
+    Returns the new ctx_kv (same structure; untouched requests share their arrays with the input)."""
+    out = list(ctx_kv)
+    grow = [r for r in range(len(m)) if m[r] > 0]
+    if not grow:
+        return out
+    toks = [np.concatenate([np.asarray(draft_steps[req_offsets[r] + j]) for j in range(int(m[r]))]) for r in grow]
+    lens = [ctx_kv[r][0][0].shape[0] for r in grow]
+    _, new = forward_extend(weights, toks, lens, lambda j, l: ctx_kv[grow[j]][l], collect_new_kv=True)
+    for j, r in enumerate(grow):
+        layers = []
+        for l, (k, v) in enumerate(new[j]):
+            if store_bf16:
+                k, v = round_to_bf16(k), round_to_bf16(v)
+            layers.append((np.concatenate([ctx_kv[r][l][0], k], axis=0), np.concatenate([ctx_kv[r][l][1], v], axis=0)))
+        out[r] = layers
+    return out

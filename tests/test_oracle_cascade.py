@@ -94,3 +94,32 @@ def test_single_escalated_step_uses_its_own_context(two_models):
     assert np.max(np.abs(r["target"]["logits"][0] - full_t["logits"][lowest])) < 1e-9
     others = [i for i in range(b.n_steps) if i != lowest]
     assert min(np.max(np.abs(full_t["logits"][i] - full_t["logits"][lowest])) for i in others) > 1e-3
+
+
+def test_appending_accepted_steps_equals_prefilling_the_longer_context():
+    """Stage 3 of Algorithm 1 in terms of the cache: context (+) accepted steps, built by appending, is the cache a
+    prefill of the concatenated tokens builds from nothing; a request with m = 0 keeps its cache."""
+    cfg = get_config("cfg1_tiny")
+    w = model_weights(cfg.model, cfg.seed)
+    g = np.random.default_rng(9)
+    V = cfg.model.vocab
+    ctx = [g.integers(3, V, size=n).astype(np.int32) for n in (19, 33, 7)]
+    req_offsets = [0, 3, 5, 8]                                   # 3, 2 and 3 candidate steps
+    steps = [g.integers(3, V, size=n).astype(np.int32) for n in (4, 9, 2, 5, 5, 1, 6, 3)]
+    m = [2, 0, 3]
+    kv = O.prefill_context(w, ctx, store_bf16=False)
+    new = O.append_accepted_steps(w, kv, m, req_offsets, steps, store_bf16=False)
+    longer = [np.concatenate([ctx[0], steps[0], steps[1]]), ctx[1], np.concatenate([ctx[2], steps[5], steps[6], steps[7]])]
+    want = O.prefill_context(w, longer, store_bf16=False)
+    for r in range(3):
+        for l in range(cfg.model.n_layers):
+            for a, b in zip(new[r][l], want[r][l]):
+                assert a.shape == b.shape and np.max(np.abs(a - b)) < 1e-10
+    assert new[1] is kv[1]
+    assert new[0][0][0].shape[0] == 19 + 4 + 9 and new[2][1][1].shape[0] == 7 + 1 + 6 + 3
+    # cache format: the appended rows are bf16 values, the earlier rows are the earlier bits
+    kvb = O.prefill_context(w, ctx, store_bf16=True)
+    newb = O.append_accepted_steps(w, kvb, m, req_offsets, steps, store_bf16=True)
+    k_new = newb[0][1][0]
+    assert np.array_equal(k_new[:19], kvb[0][1][0]) and np.array_equal(O.round_to_bf16(k_new), k_new)
+    assert np.max(np.abs(k_new[19:] - new[0][1][0][19:])) < 0.05 and np.max(np.abs(k_new[19:] - new[0][1][0][19:])) > 0
