@@ -140,6 +140,33 @@ int cs_prefill(cs_model* model, cs_kv* kv, const int32_t* seq_ids, const int32_t
                const int32_t* lens, int B, void* stream);
 
 /*
+ * cs_append_accepted - context management of Algorithm 1, Stage 3, in terms of the cache: for every request r whose
+ * accept-prefix length m_r (out_prefix_len of cs_cascade_select) is positive,
+ *     context_r <- context_r (+) s^_1 (+) ... (+) s^_m,
+ * i.e. the tokens of its first m_r drafted steps run through the model on top of the cached context and their K/V
+ * are appended to the pages of the request's sequence (one cs_prefill over all such requests). Requests with
+ * m_r = 0 are left alone: their next step comes from the target model's generation, which is outside this library.
+ * The k candidates of a request are verified on the request's own sequence id (cs_verify_steps takes the same
+ * sequence several times), so they share its pages; nothing is copied per candidate, and after this call the next
+ * iteration's candidates see the longer context under the same id.
+ *   kv                 cache of `model`; call once per model that caches the contexts (draft and target).
+ *   req_seq_ids        host int32[R], distinct: the sequence holding request r's context. It must already own
+ *                      pages for the appended tokens (cs_kv_set_seq), else CS_EINVAL and nothing is appended.
+ *   req_offsets        host int32[R + 1]: the steps of request r are [req_offsets[r], req_offsets[r+1]) of the batch.
+ *   dev_prefix_len     DEVICE int32[R], each in [0, number of steps of the request]; read back inside the call
+ *                      (4 R bytes, blocks the host once).
+ *   step_tokens, step_lens   host, as given to cs_verify_steps (the whole verification spans).
+ *   draft_lens         host int32[B]: how many leading tokens of span i are the drafted step s^_i itself
+ *                      (0 <= draft_lens[i] <= step_lens[i]); the rest of the span (the target's step, the
+ *                      verification prompt) never enters the context.
+ *   host_prefix_len    host int32[R] or NULL: receives the m_r that were read.
+ * Errors: CS_EINVAL, CS_ESTATE (unset sequence) before any launch; then as cs_prefill.
+ */
+int cs_append_accepted(cs_model* model, cs_kv* kv, int R, const int32_t* req_seq_ids, const int32_t* req_offsets,
+                       const int32_t* dev_prefix_len, const int32_t* step_tokens, const int32_t* step_lens,
+                       const int32_t* draft_lens, int32_t* host_prefix_len, void* stream);
+
+/*
  * cs_verify_steps — the verification pass itself (M.verify of Algorithm 1, Stage 2; Eqs. 2-4).
  * For step i, the new tokens step_tokens[cu[i] .. cu[i]+step_lens[i]) (draft step, target step and the
  * verification prompt, as one opaque span) are placed at positions ctx_len .. ctx_len+step_lens[i]-1 after

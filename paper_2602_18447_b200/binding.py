@@ -16,7 +16,7 @@ CS_OK, CS_EINVAL, CS_ENOMEM, CS_ECUDA, CS_ETIMEOUT, CS_ESTATE, CS_ELIMIT = range
 EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_reserve",
     "cs_kv_alloc", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
-    "cs_verify_steps", "cs_verify_cascade", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
+    "cs_verify_steps", "cs_verify_cascade", "cs_append_accepted", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
     "cs_last_status", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
 ]
 
@@ -74,6 +74,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_prefill": (C.c_int, [vp, vp, vp, vp, vp, i32, vp]),
         "cs_verify_steps": (C.c_int, [vp, vp, vp, i32, vp, i32, vp, vp, i32, f32, vp, vp, vp, vp]),
         "cs_verify_cascade": (C.c_int, [vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
+        "cs_append_accepted": (C.c_int, [vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
         "cs_escalate_mask": (C.c_int, [vp, i32, f32, vp, vp, vp, vp]),
         "cs_cascade_select": (C.c_int, [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]),
         "cs_set_keep_logits": (C.c_int, [vp, i32]),
@@ -254,6 +255,20 @@ def cs_verify_cascade(draft: int, kv_d: int, target: int, kv_t: int, seq_ids, st
                                             _dev_ptr(out_verdict_t), _dev_ptr(out_verdict), _dev_ptr(out_conf),
                                             C.cast(C.byref(n_esc), C.c_void_p), _stream_ptr(stream)), "cs_verify_cascade")
     return int(n_esc.value)
+
+
+def cs_append_accepted(model: int, kv: int, req_seq_ids, req_offsets, prefix_len, step_tokens, step_lens, draft_lens,
+                       stream=None) -> np.ndarray:
+    """prefix_len: CUDA int32 tensor [R] (out_prefix_len of cs_cascade_select); the other arrays are host int32.
+    Returns the prefix lengths that were read back."""
+    q, o, t = _i32(req_seq_ids), _i32(req_offsets), _i32(step_tokens)
+    l, d = _i32(step_lens), _i32(draft_lens)
+    R = int(q.shape[0])
+    got = np.zeros(max(R, 1), dtype=np.int32)
+    _check(load_library().cs_append_accepted(model, kv, R, _np_ptr(q), _np_ptr(o), _dev_ptr(prefix_len), _np_ptr(t),
+                                             _np_ptr(l), _np_ptr(d), _np_ptr(got), _stream_ptr(stream)),
+           "cs_append_accepted")
+    return got[:R]
 
 
 def cs_escalate_mask(conf, tau: float, out_accept, out_escalate_idx, out_escalate_count, stream=None) -> None:

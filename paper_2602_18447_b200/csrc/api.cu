@@ -156,6 +156,18 @@ int staging_slot(Staging& st, size_t ints, int* slot_out) {
   return CS_OK;
 }
 
+// Pinned host buffer of at least `ints` int32 for small device-to-host read-backs.
+int ensure_readback(cs_model* m, size_t ints) {
+  if (m->casc_host_cap >= ints) return CS_OK;
+  if (m->casc_host) cudaFreeHost(m->casc_host);
+  m->casc_host = nullptr;
+  m->casc_host_cap = 0;
+  const size_t want = 2 * ints + 64;
+  CS_CUDA(cudaMallocHost(reinterpret_cast<void**>(&m->casc_host), want * sizeof(int32_t)));
+  m->casc_host_cap = want;
+  return CS_OK;
+}
+
 struct BatchLayout {
   int B = 0, T = 0;
   size_t off_cu, off_pos, off_tseq, off_tok, off_items, total;
@@ -756,6 +768,51 @@ int cs_prefill(cs_model* m, cs_kv* kv, const int32_t* seq_ids, const int32_t* to
   return CS_OK;
 }
 
+int cs_append_accepted(cs_model* m, cs_kv* kv, int R, const int32_t* req_seq_ids, const int32_t* req_offsets,
+                       const int32_t* dev_prefix_len, const int32_t* step_tokens, const int32_t* step_lens,
+                       const int32_t* draft_lens, int32_t* host_prefix_len, void* stream) {
+  if (!m || !kv || kv->model != m || R < 0) return CS_EINVAL;
+  if (R == 0) return CS_OK;
+  if (!req_seq_ids || !req_offsets || !dev_prefix_len || !step_tokens || !step_lens || !draft_lens) return CS_EINVAL;
+  if (req_offsets[0] != 0) return CS_EINVAL;
+  for (int r = 0; r < R; ++r) {
+    if (req_offsets[r + 1] < req_offsets[r]) return CS_EINVAL;
+    if (req_seq_ids[r] < 0 || req_seq_ids[r] >= kv->max_seqs) return CS_EINVAL;
+    if (kv->ctx_len[req_seq_ids[r]] < 0) return CS_ESTATE;
+    for (int q = 0; q < r; ++q)
+      if (req_seq_ids[q] == req_seq_ids[r]) return CS_EINVAL;
+  }
+  const int B = req_offsets[R];
+  std::vector<int64_t> cu(static_cast<size_t>(B) + 1, 0);
+  for (int i = 0; i < B; ++i) {
+    if (step_lens[i] < 1 || draft_lens[i] < 0 || draft_lens[i] > step_lens[i]) return CS_EINVAL;
+    cu[i + 1] = cu[i] + step_lens[i];
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc;
+  if ((rc = ensure_readback(m, static_cast<size_t>(R)))) return rc;
+  CS_CUDA(cudaMemcpyAsync(m->casc_host, dev_prefix_len, sizeof(int32_t) * R, cudaMemcpyDeviceToHost, s));
+  CS_CUDA(cudaStreamSynchronize(s));
+  std::vector<int32_t> seqs, lens, toks;
+  for (int r = 0; r < R; ++r) {
+    const int mr = m->casc_host[r];
+    if (mr < 0 || mr > req_offsets[r + 1] - req_offsets[r]) return CS_EINVAL;
+    if (host_prefix_len) host_prefix_len[r] = mr;
+    int n = 0;
+    for (int j = 0; j < mr; ++j) {
+      const int i = req_offsets[r] + j;
+      toks.insert(toks.end(), step_tokens + cu[i], step_tokens + cu[i] + draft_lens[i]);
+      n += draft_lens[i];
+    }
+    if (n > 0) {
+      seqs.push_back(req_seq_ids[r]);
+      lens.push_back(n);
+    }
+  }
+  if (seqs.empty()) return CS_OK;
+  return cs_prefill(m, kv, seqs.data(), toks.data(), lens.data(), static_cast<int>(seqs.size()), stream);
+}
+
 int cs_verify_steps(cs_model* m, const cs_kv* ckv, const int32_t* seq_ids, int B, const int32_t* step_tokens,
                     int tokens_on_device, const int32_t* step_lens, const int32_t* verdict_ids, int n_verdict,
                     float tau, float* out_conf, uint8_t* out_accept, int32_t* out_verdict, void* stream) {
@@ -843,14 +900,7 @@ int cs_verify_cascade(cs_model* draft, const cs_kv* kv_d, cs_model* target, cons
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int rc;
   if ((rc = draft->casc_idx.ensure(sizeof(int32_t) * (static_cast<size_t>(B) + 1)))) return rc;
-  if (draft->casc_host_cap < static_cast<size_t>(B) + 1) {
-    if (draft->casc_host) cudaFreeHost(draft->casc_host);
-    draft->casc_host = nullptr;
-    draft->casc_host_cap = 0;
-    const size_t want = 2 * static_cast<size_t>(B) + 64;
-    CS_CUDA(cudaMallocHost(reinterpret_cast<void**>(&draft->casc_host), want * sizeof(int32_t)));
-    draft->casc_host_cap = want;
-  }
+  if ((rc = ensure_readback(draft, static_cast<size_t>(B) + 1))) return rc;
   // tier 1: every step through the draft model
   if ((rc = cs_verify_steps(draft, kv_d, seq_ids, B, step_tokens, 0, step_lens, verdict_ids, n_verdict, tau, out_conf_d,
                             out_trusted, out_verdict_d, stream)))
