@@ -24,7 +24,8 @@ attention with scalar loops, cache-extend == full causal recompute, rotary
 shift invariance, GQA == MHA with repeated heads, softmax sums to one, gate
 end points of Table 3 (gamma = 0 never escalates, gamma > 1 always does),
 batch-permutation equivariance, the whole forward against the
-`transformers` Qwen2 architecture used as a black-box library routine, and hand-worked iterations of
+`transformers` Qwen2 architecture (and, with per-head query/key normalisation, its Qwen3 architecture) used
+as a black-box library routine, and hand-worked iterations of
 Algorithm 1 / Eq. 5 for the selection bookkeeping (tests/golden/cascade_cases.txt); for the two-tier
 verifier, its reduction to one tier at either end of the threshold and the rule of Eq. 4 applied step by step
 to two independent full-batch runs; for the append of accepted steps (Stage 3), its equality with a prefill
@@ -114,6 +115,9 @@ class LayerWeights:
             setattr(self, name, widen_bf16(layer[name]))
         self.norm1 = np.asarray(layer["norm1"], dtype=np.float64)
         self.norm2 = np.asarray(layer["norm2"], dtype=np.float64)
+        # per-head RMSNorm gains of the query and key vectors ([hd] each); absent in the first model family
+        self.q_norm = np.asarray(layer["q_norm"], dtype=np.float64) if "q_norm" in layer else None
+        self.k_norm = np.asarray(layer["k_norm"], dtype=np.float64) if "k_norm" in layer else None
 
 
 def decoder_layer_extend(x: np.ndarray, lw: LayerWeights, shape, ctx_len: int,
@@ -130,6 +134,11 @@ def decoder_layer_extend(x: np.ndarray, lw: LayerWeights, shape, ctx_len: int,
     q = (a @ lw.wq.T).reshape(n, hq, hd)
     k = (a @ lw.wk.T).reshape(n, hkv, hd)
     v = (a @ lw.wv.T).reshape(n, hkv, hd)
+    if lw.q_norm is not None:
+        # second model family of the paper's experiments (Section 5.1): every head's query and key vector is
+        # RMS-normalised over its hd entries, with one gain vector shared by all heads, before the rotary turn
+        q = rmsnorm(q, lw.q_norm, shape.rms_eps)
+        k = rmsnorm(k, lw.k_norm, shape.rms_eps)
     q = rope(q, pos, shape.rope_theta)
     k = rope(k, pos, shape.rope_theta)
     o = attention_extend(q, k_ctx, v_ctx, k, v).reshape(n, hq * hd)

@@ -150,3 +150,49 @@ def test_tiny_config_runs_and_planted_rows_spread_the_confidence():
     assert r["conf"].min() < 0.3 and r["conf"].max() > 0.9      # both sides of the thresholds in use
     assert 0 < r["accept"].sum() < big.batch
     assert set(r["verdict"].tolist()) == {0, 1}
+
+
+def test_whole_forward_with_qk_norm_against_transformers_qwen3(small_case):
+    """The second model family normalises every head's query and key vector before the rotary turn; the library's
+    Qwen3 architecture, as a black box on the same weights, fixes where that norm sits and what it is taken over."""
+    torch = pytest.importorskip("torch")
+    tr = pytest.importorskip("transformers")
+    w0, ctx, new = small_case
+    m = SMALL
+    g = np.random.default_rng(21)
+    w = dict(w0, layers=[dict(l, q_norm=(1.0 + 0.3 * g.standard_normal(m.head_dim)).astype(np.float32),
+                              k_norm=(1.0 + 0.3 * g.standard_normal(m.head_dim)).astype(np.float32))
+                         for l in w0["layers"]])
+    cfg = tr.Qwen3Config(vocab_size=m.vocab, hidden_size=m.d_model, intermediate_size=m.d_ffn,
+                         num_hidden_layers=m.n_layers, num_attention_heads=m.n_q_heads,
+                         num_key_value_heads=m.n_kv_heads, head_dim=m.head_dim, rms_norm_eps=m.rms_eps,
+                         rope_theta=m.rope_theta, tie_word_embeddings=False, max_position_embeddings=4096,
+                         attn_implementation="eager", use_sliding_window=False, attention_bias=False)
+    assert cfg.rope_parameters["rope_theta"] == m.rope_theta
+    model = tr.Qwen3ForCausalLM(cfg).double().eval()
+    t = lambda bits: torch.from_numpy(O.widen_bf16(bits))
+    f = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
+    sd = {"model.embed_tokens.weight": t(w["embed"]), "lm_head.weight": t(w["lm_head"]),
+          "model.norm.weight": f(w["final_norm"])}
+    names = {"wq": "self_attn.q_proj", "wk": "self_attn.k_proj", "wv": "self_attn.v_proj",
+             "wo": "self_attn.o_proj", "wg": "mlp.gate_proj", "wu": "mlp.up_proj", "wd": "mlp.down_proj"}
+    for li, l in enumerate(w["layers"]):
+        for k, hf in names.items():
+            sd[f"model.layers.{li}.{hf}.weight"] = t(l[k])
+        sd[f"model.layers.{li}.self_attn.q_norm.weight"] = f(l["q_norm"])
+        sd[f"model.layers.{li}.self_attn.k_norm.weight"] = f(l["k_norm"])
+        sd[f"model.layers.{li}.input_layernorm.weight"] = f(l["norm1"])
+        sd[f"model.layers.{li}.post_attention_layernorm.weight"] = f(l["norm2"])
+    missing, unexpected = model.load_state_dict(sd, strict=False)
+    assert not unexpected and all("rotary" in k or "inv_freq" in k for k in missing), (missing, unexpected)
+    kv = O.prefill_context(w, ctx, store_bf16=False)
+    ours = O.verify_steps(w, new, [len(c) for c in ctx], lambda i, l: kv[i][l], (1, 2), 0.5)
+    kv0 = O.prefill_context(w0, ctx, store_bf16=False)
+    plain = O.verify_steps(w0, new, [len(c) for c in ctx], lambda i, l: kv0[i][l], (1, 2), 0.5)
+    for i in range(len(ctx)):
+        ids = torch.from_numpy(np.concatenate([ctx[i], new[i]]).astype(np.int64))[None]
+        with torch.no_grad():
+            ref = model(input_ids=ids).logits[0, -1].numpy()
+        assert np.max(np.abs(ref - ours["logits"][i])) < 1e-5
+    # the norm is not a no-op on this case
+    assert np.max(np.abs(plain["logits"] - ours["logits"])) > 0.1

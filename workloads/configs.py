@@ -26,6 +26,8 @@ class ModelShape:
     rope_theta: float
     rms_eps: float = 1e-6
     init_std: float = 0.02
+    # per-head RMSNorm of the query and key vectors before the rotary turn (the Qwen3-style second family)
+    qk_norm: bool = False
 
     @property
     def q_dim(self) -> int:

@@ -87,6 +87,12 @@ def model_weights(m: ModelShape, seed: int, threads: Optional[int] = None) -> di
                 layer[name] = _normal_bf16((seed, _TAG_WEIGHT, li + 1, ti), shapes[name], m.init_std, pool)
             layer["norm1"] = np.ones(m.d_model, dtype=np.float32)
             layer["norm2"] = np.ones(m.d_model, dtype=np.float32)
+            if m.qk_norm:
+                # trained gains of this kind are far from 1 and differ per entry; draw them so that a swapped
+                # or dropped gain shows
+                g = _rng(seed, _TAG_WEIGHT, li + 1, 100)
+                layer["q_norm"] = (1.0 + 0.25 * g.standard_normal(m.head_dim)).astype(np.float32)
+                layer["k_norm"] = (1.0 + 0.25 * g.standard_normal(m.head_dim)).astype(np.float32)
             w["layers"].append(layer)
     return w
 
