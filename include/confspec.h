@@ -63,6 +63,11 @@ typedef struct cs_model_tensors {
   const uint16_t* const* wd;    /* [d_model, d_ffn]  SwiGLU down */
   const float* const* norm1;    /* [d_model] gain of the pre-attention RMSNorm */
   const float* const* norm2;    /* [d_model] gain of the pre-MLP RMSNorm */
+  /* Second model family of the paper's experiments (Section 5.1): every head's query and key vector is
+   * RMS-normalised over its head_dim entries (eps = rms_eps) before the rotary turn, with one gain vector per layer
+   * shared by all query heads and one shared by all key heads. Both NULL: no such normalisation. */
+  const float* const* q_norm;   /* [head_dim] or NULL */
+  const float* const* k_norm;   /* [head_dim] or NULL */
 } cs_model_tensors;
 
 /* Library version as major*10000 + minor*100 + patch. */

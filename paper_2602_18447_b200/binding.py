@@ -42,7 +42,7 @@ _PP = C.POINTER(C.c_void_p)
 class cs_model_tensors(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
                 ("wq", _PP), ("wk", _PP), ("wv", _PP), ("wo", _PP), ("wg", _PP), ("wu", _PP), ("wd", _PP),
-                ("norm1", _PP), ("norm2", _PP)]
+                ("norm1", _PP), ("norm2", _PP), ("q_norm", _PP), ("k_norm", _PP)]
 
 
 _lib: Optional[C.CDLL] = None
@@ -153,6 +153,7 @@ def cs_model_load(shape, weights: dict) -> int:
     desc = cs_model_desc(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                          shape.d_ffn, shape.vocab, shape.rope_theta, shape.rms_eps)
     keep = []
+    qk = "q_norm" in weights["layers"][0]
 
     def mat(a, dtype):
         a = np.ascontiguousarray(a, dtype=dtype)
@@ -168,7 +169,8 @@ def cs_model_load(shape, weights: dict) -> int:
                          mat(weights["final_norm"], np.float32),
                          per_layer("wq", np.uint16), per_layer("wk", np.uint16), per_layer("wv", np.uint16),
                          per_layer("wo", np.uint16), per_layer("wg", np.uint16), per_layer("wu", np.uint16),
-                         per_layer("wd", np.uint16), per_layer("norm1", np.float32), per_layer("norm2", np.float32))
+                         per_layer("wd", np.uint16), per_layer("norm1", np.float32), per_layer("norm2", np.float32),
+                         per_layer("q_norm", np.float32) if qk else None, per_layer("k_norm", np.float32) if qk else None)
     out = C.c_void_p()
     _check(lib.cs_model_load(C.byref(desc), C.byref(t), 0, C.byref(out)), "cs_model_load")
     return out.value

@@ -35,6 +35,7 @@ constexpr int kStagingRing = 4;
 struct LayerDev {
   uint16_t *wqkv, *wo, *wg, *wu, *wd;
   float *norm1, *norm2;
+  float* qk_gain = nullptr;   // [2 * head_dim]: query gains then key gains; null when the family has no such norm
   CUtensorMap tm_wqkv, tm_wo, tm_wg, tm_wu, tm_wd;
 };
 
@@ -366,9 +367,12 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   ap.status = m->status;
   const int plane_groups = kv->num_pages * d.n_kv_heads * kPageSize / 8;
 
-  const RopeEpilogue rope_epi{rope, d.head_dim / 2, (d.n_q_heads + d.n_kv_heads) * d.head_dim};
+  RopeEpilogue rope_epi{rope, d.head_dim / 2, (d.n_q_heads + d.n_kv_heads) * d.head_dim};
+  rope_epi.q_cols = m->q_dim;
+  rope_epi.eps = d.rms_eps;
   for (int l = 0; l < d.n_layers; ++l) {
     const LayerDev& lw = m->layers[l];
+    rope_epi.qk_gain = lw.qk_gain;
     CS_STEP(kProfNorm, launch_rmsnorm(x, lw.norm1, a, T, d.d_model, d.rms_eps, s));
     // q and k heads leave the projection already rotated (the turn is applied to the fp32 accumulators)
     CS_STEP(kProfQkv, gemm_f16_rope(tm_a, lw.tm_wqkv, qkv, T, m->n_qkv, d.d_model, rope_epi, m->status, s));
@@ -520,6 +524,10 @@ int cs_model_load(const cs_model_desc* desc, const cs_model_tensors* t, int on_d
     if (!t->wq[l] || !t->wk[l] || !t->wv[l] || !t->wo[l] || !t->wg[l] || !t->wu[l] || !t->wd[l] || !t->norm1[l] ||
         !t->norm2[l])
       return CS_EINVAL;
+  if ((t->q_norm == nullptr) != (t->k_norm == nullptr)) return CS_EINVAL;
+  if (t->q_norm)
+    for (int l = 0; l < desc->n_layers; ++l)
+      if (!t->q_norm[l] || !t->k_norm[l]) return CS_EINVAL;
   int dev = 0;
   cudaDeviceProp prop;
   CS_CUDA(cudaGetDevice(&dev));
@@ -566,6 +574,16 @@ int cs_model_load(const cs_model_desc* desc, const cs_model_tensors* t, int on_d
     CS_TRY(dev_copy(m, &lw.wd, t->wd[l], dm * F, sd));
     CS_TRY(dev_copy(m, &lw.norm1, t->norm1[l], dm, sd));
     CS_TRY(dev_copy(m, &lw.norm2, t->norm2[l], dm, sd));
+    if (t->q_norm) {
+      void* g = nullptr;
+      e = cudaMalloc(&g, 2 * sizeof(float) * desc->head_dim);
+      if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc(qk gains)"); cs_model_free(m); return rc; }
+      m->owned.push_back(g);
+      lw.qk_gain = static_cast<float*>(g);
+      e = cudaMemcpy(lw.qk_gain, t->q_norm[l], sizeof(float) * desc->head_dim, kind);
+      if (e == cudaSuccess) e = cudaMemcpy(lw.qk_gain + desc->head_dim, t->k_norm[l], sizeof(float) * desc->head_dim, kind);
+      if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy(qk gains)"); cs_model_free(m); return rc; }
+    }
     // The matrices arrive as bf16 and are kept as fp16 (same size; see launch_bf16_to_f16): the tensor cores
     // take both operands in one 16-bit format and fp16 activations carry three more mantissa bits.
     e = launch_bf16_to_f16(lw.wqkv, static_cast<size_t>(m->n_qkv) * dm, nullptr);

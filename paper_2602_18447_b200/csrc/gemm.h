@@ -11,7 +11,8 @@ enum GemmEpilogue {
   kEpiStoreF16 = 0,  // out fp16 [M,N] = a * w^T
   kEpiResidAdd = 1,   // out fp32 [M,N] += a * w^T   (atomic adds, k-range split over the SMs)
   kEpiSwiGLU = 2,     // out fp16 [M,N] = silu(a * w^T) * (a * w2^T)
-  kEpiStoreRope = 3   // out fp16 [M,N] = a * w^T with the rotary turn applied to the leading heads (QKV projection)
+  kEpiStoreRope = 3,  // out fp16 [M,N] = a * w^T with the rotary turn applied to the leading heads (QKV projection)
+  kEpiStoreNormRope = 4   // as kEpiStoreRope, each turned head RMS-normalised over its columns first (gains qk_gain)
 };
 
 // 2D tensor map over a row-major [rows, cols] matrix of 16-bit floats (fp16, or bf16 for the kv cache);
@@ -41,10 +42,16 @@ bool make_gemm_operand_map(CUtensorMap* tm, const void* base, int rows, int k);
 // Rotary position turn fused into the store epilogue of the QKV projection: columns [0, n_rot_cols) are heads of
 // 2 * half columns in which the pair (j, j + half) of row t turns by the angle whose (cos, sin) is table[t * half + j];
 // the remaining columns (the V heads) are stored as they are. half is 32 or 64; N and n_rot_cols multiples of 2 * half.
+// With qk_gain != nullptr every turned head is first RMS-normalised over its 2 * half columns (in fp32, on the
+// accumulator): x / sqrt(mean(x^2) + eps) * g, g = qk_gain[0 .. 2 half) for heads in columns [0, q_cols) (queries)
+// and qk_gain[2 half .. 4 half) for the turned heads after them (keys).
 struct RopeEpilogue {
   const float2* table;
   int half;
   int n_rot_cols;
+  const float* qk_gain = nullptr;
+  int q_cols = 0;
+  float eps = 0.f;
 };
 cudaError_t gemm_f16_rope(const CUtensorMap& ta, const CUtensorMap& tb, void* out, int M, int N, int K,
                           const RopeEpilogue& rope, uint32_t* status, cudaStream_t stream);

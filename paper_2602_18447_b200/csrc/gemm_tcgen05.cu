@@ -273,7 +273,7 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       const bool row_ok = row < M;
       // Rotary epilogue: this row's (cos, sin) pairs are fetched while the tile is still being accumulated.
       float4 rot[32];
-      if (EPI == kEpiStoreRope && row_ok && n0 < rope.n_rot_cols) {
+      if ((EPI == kEpiStoreRope || EPI == kEpiStoreNormRope) && row_ok && n0 < rope.n_rot_cols) {
         const float4* tb = reinterpret_cast<const float4*>(rope.table + static_cast<size_t>(row) * rope.half);
 #pragma unroll
         for (int j = 0; j < 32; ++j)
@@ -305,12 +305,27 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
               if (col + j * 8 < N) st_v4(o + col + j * 8, p[4 * j], p[4 * j + 1], p[4 * j + 2], p[4 * j + 3]);
           }
         }
-      } else if (EPI == kEpiStoreRope) {
+      } else if (EPI == kEpiStoreRope || EPI == kEpiStoreNormRope) {
         __half* o = reinterpret_cast<__half*>(out) + static_cast<size_t>(row) * N;
         const int hd = 2 * rope.half;
 #pragma unroll 1
         for (int h0 = 0; h0 < BN && n0 + h0 < N; h0 += hd) {
           if (n0 + h0 < rope.n_rot_cols) {
+            // Query/key normalisation: a first sweep over the head's columns for this row's mean square.
+            float inv_rms = 1.f;
+            const float* gain = nullptr;
+            if (EPI == kEpiStoreNormRope) {
+              float ss = 0.f;
+#pragma unroll 1
+              for (int c = 0; c < hd / 32; ++c) {
+                tmem_ld_32x32(t_row + h0 + c * 32, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) ss = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ss);
+              }
+              inv_rms = rsqrtf(ss / static_cast<float>(hd) + rope.eps);
+              gain = rope.qk_gain + (n0 + h0 < rope.q_cols ? 0 : hd);
+            }
             // pairs (j, j + half) of one head, 16 pairs at a time
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -323,8 +338,16 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                   const float4 cs = rot[c * 8 + e];      // (cos, sin) of pairs 2e and 2e + 1 of this chunk
-                  const float a0 = __uint_as_float(lo[2 * e]), a1 = __uint_as_float(lo[2 * e + 1]);
-                  const float b0 = __uint_as_float(hi[2 * e]), b1 = __uint_as_float(hi[2 * e + 1]);
+                  float a0 = __uint_as_float(lo[2 * e]), a1 = __uint_as_float(lo[2 * e + 1]);
+                  float b0 = __uint_as_float(hi[2 * e]), b1 = __uint_as_float(hi[2 * e + 1]);
+                  if (EPI == kEpiStoreNormRope) {
+                    const float2 ga = __ldg(reinterpret_cast<const float2*>(gain + c * 16 + 2 * e));
+                    const float2 gb = __ldg(reinterpret_cast<const float2*>(gain + rope.half + c * 16 + 2 * e));
+                    a0 *= inv_rms * ga.x;
+                    a1 *= inv_rms * ga.y;
+                    b0 *= inv_rms * gb.x;
+                    b1 *= inv_rms * gb.y;
+                  }
                   plo[e] = pack_f16x2(a0 * cs.x - b0 * cs.y, a1 * cs.z - b1 * cs.w);
                   phi[e] = pack_f16x2(b0 * cs.x + a0 * cs.y, b1 * cs.z + a1 * cs.w);
                 }
@@ -544,6 +567,10 @@ cudaError_t gemm_f16_rope(const CUtensorMap& ta, const CUtensorMap& tb, void* ou
   if (M <= 0) return cudaSuccess;
   if (!rope.table || (rope.half != 32 && rope.half != 64) || N % (2 * rope.half) || rope.n_rot_cols % (2 * rope.half))
     return cudaErrorInvalidValue;
+  if (rope.qk_gain) {
+    if (rope.q_cols % (2 * rope.half) || rope.q_cols > rope.n_rot_cols) return cudaErrorInvalidValue;
+    return launch<256, kEpiStoreNormRope>(ta, tb, tb, out, M, N, K, status, stream, rope);
+  }
   return launch<256, kEpiStoreRope>(ta, tb, tb, out, M, N, K, status, stream, rope);
 }
 

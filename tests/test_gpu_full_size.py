@@ -102,3 +102,23 @@ def test_cfg5_7b_shape_full_depth():
     _, ses, gpu, ref, stats = _run_full("cfg5_7b_b32", None, sample=[5, 28])
     ses.close()
     assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
+
+
+@pytest.fixture(scope="module")
+def weights_q3():
+    cfg = get_config("cfg6_q3_b16")
+    return model_weights(cfg.model, cfg.seed)
+
+
+def test_cfg6_second_family_full_depth(weights_q3):
+    """The 1.7B-shaped model of the second family (query/key normalisation, 8 KV heads), all 28 layers."""
+    cfg, ses, gpu, ref, stats = _run_full("cfg6_q3_b16", weights_q3, sample=[2, 11])
+    ses.close()
+    assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
+
+
+def test_cfg7_short_steps_on_long_contexts_full_depth(weights_q3):
+    """Decode-shaped batch: 64 steps of 5 to 8 new tokens on contexts of 2K to 8K tokens."""
+    cfg, ses, gpu, ref, stats = _run_full("cfg7_q3_short", weights_q3, sample=[0, 33, 63])
+    ses.close()
+    assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL

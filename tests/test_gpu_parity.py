@@ -137,3 +137,25 @@ def test_invalid_arguments_are_rejected_before_any_launch():
         assert B.cs_take_launch_count() == 0
     finally:
         ses.close()
+
+
+def test_qk_norm_family_tiny_with_real_prefill():
+    """Per-head query/key RMSNorm before the rotary turn (fused into the QKV projection's epilogue), through a real
+    prefill and a verification pass; the planted variant puts the gate on both sides."""
+    cfg = get_config("cfg8_tiny_qknorm")
+    stats, gpu, ref = _run(cfg, model_weights(cfg.model, cfg.seed), make_batch(cfg))
+    assert stats["logit_err"] < 3e-2
+    _run(cfg, P.planted_weights(cfg), make_batch(cfg), taus=(0.5, 0.9), planted=True)
+    # the gains matter: the oracle without them is far away
+    w = model_weights(cfg.model, cfg.seed)
+    plain = dict(w, layers=[{k: v for k, v in l.items() if k not in ("q_norm", "k_norm")} for l in w["layers"]])
+    other = P.oracle_outputs(cfg, plain, make_batch(cfg))
+    assert np.max(np.abs(other["logits"] - ref["logits"])) > 10 * P.LOGIT_TOL
+
+
+@pytest.mark.parametrize("name,layers,batch", [("cfg6_q3_b16", 2, 4), ("cfg7_q3_short", 2, 9)])
+def test_qk_norm_family_reduced_depth(name, layers, batch):
+    cfg = scaled_config(name, n_layers=layers, batch=batch, vocab=20480 + 8)
+    stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), taus=(0.5,), planted=True)
+    assert stats["logit_err"] < 3e-2
+    _run(cfg, model_weights(cfg.model, cfg.seed), make_batch(cfg))

@@ -49,6 +49,9 @@ class ModelShape:
 TINY = ModelShape("tiny", 2, 256, 4, 4, 64, 688, 4096, 1.0e4)
 QWEN_1P5B = ModelShape("qwen2.5-1.5b-shaped", 28, 1536, 12, 2, 128, 8960, 151936, 1.0e6)
 QWEN_7B = ModelShape("qwen2.5-7b-shaped", 28, 3584, 28, 4, 128, 18944, 152064, 1.0e6)
+# the draft model of the paper's second family (per-head query/key normalisation, head_dim not d_model / heads)
+QWEN3_1P7B = ModelShape("qwen3-1.7b-shaped", 28, 2048, 16, 8, 128, 6144, 151936, 1.0e6, qk_norm=True)
+TINY_QKNORM = ModelShape("tiny-qknorm", 2, 256, 4, 2, 64, 688, 4096, 1.0e4, qk_norm=True)
 
 
 @dataclass(frozen=True)
@@ -84,6 +87,16 @@ CONFIGS = {
         "cfg4_1p5b_long", QWEN_1P5B, 8, ("uniform", 8192, 32768), ("uniform", 32, 128), tau=0.9, seed=404),
     "cfg5_7b_b32": VerifyConfig(
         "cfg5_7b_b32", QWEN_7B, 32, ("uniform", 1024, 4096), ("uniform", 24, 96), tau=0.9, seed=505),
+    # beyond the five: the second model family, with the first family's batch recipe ...
+    "cfg6_q3_b16": VerifyConfig(
+        "cfg6_q3_b16", QWEN3_1P7B, 16, ("uniform", 512, 2048), ("uniform", 24, 96), tau=0.9, seed=606),
+    # ... and a decode-shaped batch: many steps of at most 8 new tokens on long contexts, where attention is
+    # bound by reading the cache rather than by arithmetic
+    "cfg7_q3_short": VerifyConfig(
+        "cfg7_q3_short", QWEN3_1P7B, 64, ("uniform", 2048, 8192), ("uniform", 1, 4), suffix_len=4, tau=0.9, seed=707),
+    "cfg8_tiny_qknorm": VerifyConfig(
+        "cfg8_tiny_qknorm", TINY_QKNORM, 6, ("uniform", 20, 150), ("uniform", 1, 40), tau=0.8, ctx_kv="prefill",
+        seed=808),
 }
 
 
