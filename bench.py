@@ -36,8 +36,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) of one gate/up GEMM launch of the default workload, from the ncu capture summarised in
 # profiles/gemm_f16_cfg2_4layers.md, and the hash of the kernel source that capture was taken with. A changed kernel
 # has no counters: traffic is then reported as null.
-GATEUP_TRAFFIC = {"workload": "cfg2_1p5b_b16", "bytes": 58.657792e6 + 4.34688e6,
-                  "source": "paper_2602_18447_b200/csrc/gemm_tcgen05.cu", "sha256_16": "25b6cee4a6e08f25"}
+GATEUP_TRAFFIC = {"workload": "cfg2_1p5b_b16", "bytes": 58.654720e6 + 4.816128e6,
+                  "source": "paper_2602_18447_b200/csrc/gemm_tcgen05.cu", "sha256_16": "14d933d57643dc3b"}
 
 
 def gateup_traffic(workload: str):
