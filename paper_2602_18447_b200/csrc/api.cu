@@ -224,9 +224,13 @@ void build_attention_work(const cs_model* m, int B, const int32_t* lens, const i
   }
   const int heads = m->d.n_kv_heads;
   auto pieces = [&](int nt, int cap) { return std::min(max_splits, (nt + cap - 1) / cap); };
-  auto estimate = [&](int cap) {
-    std::vector<double> cost;
-    cost.reserve(units.size() * heads * 2);
+  // No schedule finishes before its longest item or before the work divided by the SMs: a candidate whose bound
+  // cannot beat `to_beat` is dropped without being scheduled (the call runs on the host before the first launch).
+  std::vector<double> cost;
+  cost.reserve(units.size() * heads * 2);
+  auto estimate = [&](int cap, double to_beat) {
+    cost.clear();
+    double longest_item = 0.0, total = 0.0;
     for (const Unit& u : units) {
       const int n = pieces(u.nt, cap);
       for (int s = 0; s < n; ++s) {
@@ -235,17 +239,21 @@ void build_attention_work(const cs_model* m, int B, const int32_t* lens, const i
         if (n > 1) c += kAttnPieceExtra;
         if (n > 1 && s == n - 1) c += kAttnMergeFixed + kAttnMergePerSplit * n;
         for (int h = 0; h < heads; ++h) cost.push_back(c);
+        longest_item = std::max(longest_item, c);
+        total += c * heads;
       }
     }
+    if (static_cast<int>(cost.size()) <= kNumSMs) return longest_item;
+    if (std::max(longest_item, total / kNumSMs) >= to_beat) return to_beat;
     return list_schedule_makespan(cost, kNumSMs);
   };
   int best_cap = longest;
-  double best = estimate(longest);
+  double best = estimate(longest, 1e300);
   int last_cap = longest;
   auto consider = [&](int cap) {
     if (cap < 2 || cap >= last_cap) return;
     last_cap = cap;
-    const double e = estimate(cap);
+    const double e = estimate(cap, 0.97 * best);
     if (e < 0.97 * best) { best = e; best_cap = cap; }
   };
   // caps just below the longest range cut only the few longest query tiles (in two) ...
