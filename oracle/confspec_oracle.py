@@ -296,10 +296,17 @@ def verify_steps(weights: dict, tokens_per_step: List[np.ndarray], ctx_lens: Seq
 
 def verify_cascade(weights_d: dict, weights_t: dict, tokens_per_step: List[np.ndarray],
                    ctx_lens: Sequence[int], ctx_kv_fn_d, ctx_kv_fn_t,
-                   verdict_ids: Sequence[int], tau: float) -> dict:
+                   verdict_ids: Sequence[int], tau: float,
+                   req_offsets: Optional[Sequence[int]] = None, accept_index: int = 0) -> dict:
     """The two-tier verifier V_cascade (Eq. 4; Algorithm 1, Stage 2): every step goes through the draft
     model; the steps whose draft confidence is below gamma, and only those, go through the target model;
     the final decision of a step is r_D where p_D >= gamma and r_T otherwise.
+
+    With `req_offsets` (linear drafting: the steps of request r are req_offsets[r] .. req_offsets[r+1]-1, in
+    drafting order) the loop of Algorithm 1 over a request's steps ends at the first rejection, so a step that
+    follows a TRUSTED draft rejection in its request is never looked at again: such a step is not sent to the
+    target model even if its own confidence is below gamma, and it has no final decision (verdict -1,
+    confidence 0). Steps after an escalated step stay in, since the target may still accept that step.
 
     ctx_kv_fn_d / ctx_kv_fn_t (step, layer) -> (K, V): the same reasoning context as cached by each model,
     indexed by the step's position in the full batch.
@@ -308,9 +315,21 @@ def verify_cascade(weights_d: dict, weights_t: dict, tokens_per_step: List[np.nd
     step indices), and per step of the batch "verdict" (final decision) and "conf" (confidence of the
     verifier whose decision was taken)."""
     draft = verify_steps(weights_d, tokens_per_step, ctx_lens, ctx_kv_fn_d, verdict_ids, tau)
-    escalated = [i for i in range(len(tokens_per_step)) if not draft["accept"][i]]
+    B = len(tokens_per_step)
+    live = [True] * B
+    if req_offsets is not None:
+        for r in range(len(req_offsets) - 1):
+            alive = True
+            for i in range(int(req_offsets[r]), int(req_offsets[r + 1])):
+                live[i] = alive
+                if draft["accept"][i] and draft["verdict"][i] != accept_index:
+                    alive = False            # the loop over this request's steps breaks here
+    escalated = [i for i in range(B) if not draft["accept"][i] and live[i]]
     verdict = np.array(draft["verdict"], dtype=np.int32)
     conf = np.array(draft["conf"], dtype=np.float64)
+    for i in range(B):
+        if not draft["accept"][i]:
+            verdict[i], conf[i] = -1, 0.0
     target = None
     if escalated:
         target = verify_steps(weights_t, [tokens_per_step[i] for i in escalated],

@@ -123,3 +123,44 @@ def test_appending_accepted_steps_equals_prefilling_the_longer_context():
     k_new = newb[0][1][0]
     assert np.array_equal(k_new[:19], kvb[0][1][0]) and np.array_equal(O.round_to_bf16(k_new), k_new)
     assert np.max(np.abs(k_new[19:] - new[0][1][0][19:])) < 0.05 and np.max(np.abs(k_new[19:] - new[0][1][0][19:])) > 0
+
+
+def test_steps_behind_a_trusted_rejection_are_not_escalated_and_m_does_not_change(two_models):
+    """Linear drafting: Algorithm 1's loop over a request's steps breaks at the first rejection, so the target model
+    never needs the steps behind a trusted draft rejection. Leaving them out must not change any accept-prefix
+    length m, and must leave out exactly those steps."""
+    cfg, b, wd, wt, fd, ft, full_d, full_t = two_models
+    req_offsets = [0, 5, 8, 12]
+    n_pruned = 0
+    for tau in (0.05, 0.2, 0.5, 0.8):
+        allv = O.verify_cascade(wd, wt, _steps(b), b.ctx_lens, fd, ft, cfg.verdict_ids, tau)
+        live = O.verify_cascade(wd, wt, _steps(b), b.ctx_lens, fd, ft, cfg.verdict_ids, tau, req_offsets=req_offsets)
+        trusted, vd = allv["draft"]["accept"], allv["draft"]["verdict"]
+        expect = []
+        for r in range(3):
+            seen_reject = False
+            for i in range(req_offsets[r], req_offsets[r + 1]):
+                if not trusted[i] and not seen_reject:
+                    expect.append(i)
+                if trusted[i] and vd[i] != 0:
+                    seen_reject = True
+        assert live["escalated"].tolist() == expect
+        assert set(expect) <= set(allv["escalated"].tolist())
+        n_pruned += len(allv["escalated"]) - len(expect)
+
+        def m_of(res):
+            vt = np.full(b.n_steps, -1, np.int32)
+            ct = np.zeros(b.n_steps, np.float32)
+            if res["target"] is not None:
+                vt[res["escalated"]], ct[res["escalated"]] = res["target"]["verdict"], res["target"]["conf"]
+            return O.cascade_select(trusted, vd, allv["draft"]["conf"], vt, ct, req_offsets, accept_index=0)[2]
+
+        assert np.array_equal(m_of(allv), m_of(live))
+        for i in range(b.n_steps):
+            if trusted[i]:
+                assert live["verdict"][i] == vd[i]
+            elif i in expect:
+                assert live["verdict"][i] == allv["verdict"][i] and abs(live["conf"][i] - allv["conf"][i]) < 1e-12
+            else:
+                assert live["verdict"][i] == -1 and live["conf"][i] == 0.0
+    assert n_pruned > 0                                  # the rule left something out on this case
