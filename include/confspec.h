@@ -224,11 +224,20 @@ int cs_escalate_mask(const float* conf, int B, float tau, uint8_t* out_accept,
  *                      the host from the list of escalated steps).
  *   out_conf_d, out_trusted, out_verdict_d   device float[B], uint8[B], int32[B]: the draft tier's p_D,
  *                      (p_D >= tau), r_D as an index into verdict_ids. All required.
- *   out_conf_t, out_verdict_t   device float[B], int32[B] or NULL: the target tier's p_T and r_T at the escalated
- *                      steps, (0, -1) at the trusted ones.
+ *   out_conf_t, out_verdict_t   device float[B], int32[B] or NULL: the target tier's p_T and r_T at the steps it
+ *                      verified, (0, -1) at all others.
  *   out_verdict, out_conf   device int32[B], float[B]: final decision and the confidence of the verifier that
  *                      took it. Required.
- *   host_n_escalated   host int32[1] or NULL: number of escalated steps, valid on return.
+ *   req_offsets, R, accept_index   linear drafting (Algorithm 1): host int32[R + 1], the steps of request r are
+ *                      [req_offsets[r], req_offsets[r+1]) of the batch in drafting order, req_offsets[R] == B;
+ *                      accept_index = index into verdict_ids of the "accept" decision. The loop of Algorithm 1 over a
+ *                      request's steps breaks at the first rejection, so a step behind a TRUSTED draft rejection
+ *                      of its request is not sent to the target model even when its own confidence is below tau;
+ *                      it ends with out_verdict = -1, out_conf = 0 (cs_cascade_select counts it as rejected,
+ *                      which leaves every accept-prefix length as it would be with all steps verified).
+ *                      req_offsets == NULL (tree drafting, Section 4.3: every candidate counts): every step
+ *                      below tau goes to the target; R and accept_index are ignored.
+ *   host_n_escalated   host int32[1] or NULL: number of steps sent to the target model, valid on return.
  * The call blocks the host once between the tiers (it reads the list back: 4 (B + 1) bytes); the target pass and
  * the final scatter are asynchronous on `stream`. Arguments are checked for both tiers before anything is
  * launched. B <= 65536.
@@ -239,7 +248,7 @@ int cs_verify_cascade(cs_model* draft, const cs_kv* kv_d, cs_model* target, cons
                       const int32_t* verdict_ids, int n_verdict, float tau,
                       float* out_conf_d, uint8_t* out_trusted, int32_t* out_verdict_d,
                       float* out_conf_t, int32_t* out_verdict_t, int32_t* out_verdict, float* out_conf,
-                      int32_t* host_n_escalated, void* stream);
+                      const int32_t* req_offsets, int R, int accept_index, int32_t* host_n_escalated, void* stream);
 
 /*
  * cs_cascade_select - what the drafting loop does with the verification results of one iteration, on the device.

@@ -73,7 +73,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_kv_fill": (C.c_int, [vp, i32, i32, vp, vp, vp]),
         "cs_prefill": (C.c_int, [vp, vp, vp, vp, vp, i32, vp]),
         "cs_verify_steps": (C.c_int, [vp, vp, vp, i32, vp, i32, vp, vp, i32, f32, vp, vp, vp, vp]),
-        "cs_verify_cascade": (C.c_int, [vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
+        "cs_verify_cascade": (C.c_int, [vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp, vp, vp, vp, i32,
+                                        i32, vp, vp]),
         "cs_append_accepted": (C.c_int, [vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
         "cs_escalate_mask": (C.c_int, [vp, i32, f32, vp, vp, vp, vp]),
         "cs_cascade_select": (C.c_int, [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]),
@@ -239,9 +240,10 @@ def cs_verify_steps(model: int, ctx_kv: int, seq_ids, step_tokens, step_lens, ve
 
 def cs_verify_cascade(draft: int, kv_d: int, target: int, kv_t: int, seq_ids, step_tokens, step_lens,
                       verdict_ids: Sequence[int], tau: float, out_conf_d, out_trusted, out_verdict_d, out_conf_t,
-                      out_verdict_t, out_verdict, out_conf, stream=None) -> int:
+                      out_verdict_t, out_verdict, out_conf, req_offsets=None, accept_index: int = 0, stream=None) -> int:
     """step_tokens: host int32 (numpy or a CPU torch tensor). The out_* are CUDA tensors of length B (out_conf_t and
-    out_verdict_t may be None). Returns the number of escalated steps."""
+    out_verdict_t may be None). req_offsets (host int32 [R+1]) turns on the linear-drafting rule. Returns the number
+    of steps sent to the target model."""
     s, l, v = _i32(seq_ids), _i32(step_lens), _i32(verdict_ids)
     if hasattr(step_tokens, "is_cuda"):
         if step_tokens.is_cuda:
@@ -251,11 +253,14 @@ def cs_verify_cascade(draft: int, kv_d: int, target: int, kv_t: int, seq_ids, st
         step_tokens = _i32(step_tokens)
         tok_ptr = _np_ptr(step_tokens)
     n_esc = C.c_int32(0)
+    ro = None if req_offsets is None else _i32(req_offsets)
     _check(load_library().cs_verify_cascade(draft, kv_d, target, kv_t, _np_ptr(s), int(s.shape[0]), tok_ptr, _np_ptr(l),
                                             _np_ptr(v), int(v.shape[0]), float(tau), _dev_ptr(out_conf_d),
                                             _dev_ptr(out_trusted), _dev_ptr(out_verdict_d), _dev_ptr(out_conf_t),
                                             _dev_ptr(out_verdict_t), _dev_ptr(out_verdict), _dev_ptr(out_conf),
-                                            C.cast(C.byref(n_esc), C.c_void_p), _stream_ptr(stream)), "cs_verify_cascade")
+                                            None if ro is None else _np_ptr(ro), 0 if ro is None else int(ro.shape[0]) - 1,
+                                            int(accept_index), C.cast(C.byref(n_esc), C.c_void_p), _stream_ptr(stream)),
+           "cs_verify_cascade")
     return int(n_esc.value)
 
 

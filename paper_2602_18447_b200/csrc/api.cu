@@ -899,13 +899,19 @@ int cs_verify_cascade(cs_model* draft, const cs_kv* kv_d, cs_model* target, cons
                       int B, const int32_t* step_tokens, const int32_t* step_lens, const int32_t* verdict_ids,
                       int n_verdict, float tau, float* out_conf_d, uint8_t* out_trusted, int32_t* out_verdict_d,
                       float* out_conf_t, int32_t* out_verdict_t, int32_t* out_verdict, float* out_conf,
-                      int32_t* host_n_escalated, void* stream) {
+                      const int32_t* req_offsets, int R, int accept_index, int32_t* host_n_escalated, void* stream) {
   if (!draft || !target || draft == target || !kv_d || !kv_t || kv_d->model != draft || kv_t->model != target || B < 0)
     return CS_EINVAL;
   if (tau != tau || n_verdict < 1 || n_verdict > 8 || !verdict_ids) return CS_EINVAL;
   for (int j = 0; j < n_verdict; ++j)
     if (verdict_ids[j] < 0 || verdict_ids[j] >= draft->d.vocab || verdict_ids[j] >= target->d.vocab) return CS_EINVAL;
   if (host_n_escalated) *host_n_escalated = 0;
+  if (req_offsets) {
+    if (R < 0 || accept_index < 0 || accept_index >= n_verdict || req_offsets[0] != 0 || req_offsets[R] != B)
+      return CS_EINVAL;
+    for (int r = 0; r < R; ++r)
+      if (req_offsets[r + 1] < req_offsets[r]) return CS_EINVAL;
+  }
   if (B == 0) return CS_OK;
   if (B > 65536) return CS_EINVAL;
   if (!seq_ids || !step_tokens || !step_lens || !out_conf_d || !out_trusted || !out_verdict_d || !out_verdict ||
@@ -925,16 +931,25 @@ int cs_verify_cascade(cs_model* draft, const cs_kv* kv_d, cs_model* target, cons
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int rc;
-  if ((rc = draft->casc_idx.ensure(sizeof(int32_t) * (static_cast<size_t>(B) + 1)))) return rc;
-  if ((rc = ensure_readback(draft, static_cast<size_t>(B) + 1))) return rc;
+  if ((rc = draft->casc_idx.ensure(sizeof(int32_t) * (2 * static_cast<size_t>(B) + 1)))) return rc;
+  if ((rc = ensure_readback(draft, 2 * static_cast<size_t>(B) + 1))) return rc;
+  int32_t* idx = static_cast<int32_t*>(draft->casc_idx.p);
+  int32_t* count = idx + B;
+  int32_t* req_start = nullptr;
+  if (req_offsets) {
+    // first step of each step's request, for the rule that closes a request at a trusted rejection
+    req_start = count + 1;
+    int32_t* h = draft->casc_host + B + 1;
+    for (int r = 0; r < R; ++r)
+      for (int i = req_offsets[r]; i < req_offsets[r + 1]; ++i) h[i] = req_offsets[r];
+    CS_CUDA(cudaMemcpyAsync(req_start, h, sizeof(int32_t) * B, cudaMemcpyHostToDevice, s));
+  }
   // tier 1: every step through the draft model
   if ((rc = cs_verify_steps(draft, kv_d, seq_ids, B, step_tokens, 0, step_lens, verdict_ids, n_verdict, tau, out_conf_d,
                             out_trusted, out_verdict_d, stream)))
     return rc;
   // the steps it is not confident about, listed on the device; the host needs the list to lay out the second batch
-  int32_t* idx = static_cast<int32_t*>(draft->casc_idx.p);
-  int32_t* count = idx + B;
-  CS_CUDA(launch_escalate(out_conf_d, B, tau, nullptr, idx, count, s));
+  CS_CUDA(launch_escalate(out_conf_d, B, tau, nullptr, idx, count, s, out_verdict_d, req_start, accept_index));
   CS_CUDA(cudaMemcpyAsync(draft->casc_host + B, count, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
   CS_CUDA(cudaMemcpyAsync(draft->casc_host, idx, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
   CS_CUDA(cudaStreamSynchronize(s));

@@ -90,8 +90,10 @@ cudaError_t launch_cascade_select(const uint8_t* trusted, const int32_t* verdict
                                   const int32_t* verdict_t, const float* conf_t, const int32_t* req_offsets, int R,
                                   int accept_index, int32_t* out_prefix_len, int32_t* out_best, uint8_t* out_pass,
                                   float* out_conf, cudaStream_t s);
+// verdict_d / req_start non-null: steps behind a trusted rejection of their request are not listed (see the kernel).
 cudaError_t launch_escalate(const float* conf, int B, float tau, uint8_t* out_accept, int32_t* out_idx,
-                            int32_t* out_count, cudaStream_t s);
+                            int32_t* out_count, cudaStream_t s, const int32_t* verdict_d = nullptr,
+                            const int32_t* req_start = nullptr, int accept_index = 0);
 // Results of the target pass (compact, over the escalated steps idx[0 .. *count)) back to batch order, and the
 // final decision of Eq. 4 for every step.
 cudaError_t launch_cascade_scatter(int B, const uint8_t* trusted, const int32_t* verdict_d, const float* conf_d,

@@ -289,8 +289,13 @@ __global__ void gate_kernel(const float* __restrict__ part_max, const float* __r
 }
 
 // Single CTA: flags, then an ordered compaction of the escalated indices by a block-wide scan.
+// With req_start (linear drafting; req_start[i] = first step of step i's request) a step is listed only while its
+// request is still open: Algorithm 1's loop over a request's steps breaks at the first rejection, so a step behind a
+// trusted draft rejection (conf >= tau and verdict != accept_index at an earlier step of the request) is left out.
 __global__ void escalate_kernel(const float* __restrict__ conf, int B, float tau, uint8_t* __restrict__ out_accept,
-                                int32_t* __restrict__ out_idx, int32_t* __restrict__ out_count) {
+                                int32_t* __restrict__ out_idx, int32_t* __restrict__ out_count,
+                                const int32_t* __restrict__ verdict_d, const int32_t* __restrict__ req_start,
+                                int accept_index) {
   __shared__ int warp_tot[32];
   __shared__ int base;
   if (threadIdx.x == 0) base = 0;
@@ -303,6 +308,10 @@ __global__ void escalate_kernel(const float* __restrict__ conf, int B, float tau
       const int acc = (conf[i] >= tau) ? 1 : 0;
       if (out_accept) out_accept[i] = static_cast<uint8_t>(acc);
       esc = 1 - acc;
+      if (esc && req_start) {
+        for (int j = req_start[i]; j < i; ++j)
+          if (conf[j] >= tau && verdict_d[j] != accept_index) { esc = 0; break; }
+      }
     }
     const unsigned ball = __ballot_sync(0xffffffffu, esc);
     const int before = __popc(ball & ((1u << lane) - 1u));
@@ -503,8 +512,9 @@ cudaError_t launch_cascade_scatter(int B, const uint8_t* trusted, const int32_t*
 }
 
 cudaError_t launch_escalate(const float* conf, int B, float tau, uint8_t* out_accept, int32_t* out_idx,
-                            int32_t* out_count, cudaStream_t s) {
-  escalate_kernel<<<1, 1024, 0, s>>>(conf, B, tau, out_accept, out_idx, out_count);
+                            int32_t* out_count, cudaStream_t s, const int32_t* verdict_d, const int32_t* req_start,
+                            int accept_index) {
+  escalate_kernel<<<1, 1024, 0, s>>>(conf, B, tau, out_accept, out_idx, out_count, verdict_d, req_start, accept_index);
   count_launch();
   return cudaGetLastError();
 }

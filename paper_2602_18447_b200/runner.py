@@ -115,12 +115,13 @@ class CascadeSession:
         self.out_verdict = torch.empty(n, dtype=torch.int32, device=dev)
         self.n_escalated = -1
 
-    def verify(self, tau: Optional[float] = None, stream=None) -> int:
+    def verify(self, tau: Optional[float] = None, req_offsets=None, accept_index: int = 0, stream=None) -> int:
         d = self.draft
         self.n_escalated = B.cs_verify_cascade(
             d.model, d.kv, self.target.model, self.target.kv, d.seq_ids, d.tokens_pinned, d.batch.step_lens,
             d.cfg.verdict_ids, d.cfg.tau if tau is None else tau, d.out_conf, d.out_accept, d.out_verdict,
-            self.out_conf_t, self.out_verdict_t, self.out_verdict, self.out_conf, stream=stream)
+            self.out_conf_t, self.out_verdict_t, self.out_verdict, self.out_conf, req_offsets=req_offsets,
+            accept_index=accept_index, stream=stream)
         return self.n_escalated
 
     def results(self) -> dict:

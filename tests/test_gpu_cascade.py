@@ -113,15 +113,19 @@ def test_argument_errors_are_reported_before_any_launch():
         B.cs_take_launch_count()
 
         def call(draft=d.model, kv_d=d.kv, target=t.model, kv_t=t.kv, seq=d.seq_ids, toks=batch.step_tokens,
-                 lens=batch.step_lens, vids=cfg_d.verdict_ids, tau=0.5):
+                 lens=batch.step_lens, vids=cfg_d.verdict_ids, tau=0.5, req_offsets=None, accept_index=0):
             return B.cs_verify_cascade(draft, kv_d, target, kv_t, seq, toks, lens, vids, tau, d.out_conf, d.out_accept,
-                                       d.out_verdict, cs.out_conf_t, cs.out_verdict_t, cs.out_verdict, cs.out_conf)
+                                       d.out_verdict, cs.out_conf_t, cs.out_verdict_t, cs.out_verdict, cs.out_conf,
+                                       req_offsets=req_offsets, accept_index=accept_index)
 
         for bad in (dict(target=d.model, kv_t=d.kv),            # one model in both tiers
                     dict(kv_t=d.kv),                            # the target's cache belongs to the draft
                     dict(tau=float("nan")),
                     dict(vids=(1, cfg_t.model.vocab)),
                     dict(seq=np.full(n, n + 5, np.int32)),
+                    dict(req_offsets=np.array([0, 4, n - 1], np.int32)),     # the requests do not cover the batch
+                    dict(req_offsets=np.array([0, 7, 4, n], np.int32)),
+                    dict(req_offsets=np.array([0, n], np.int32), accept_index=2),
                     dict(lens=np.where(np.arange(n) == 3, 0, batch.step_lens).astype(np.int32)),
                     dict(toks=np.where(np.arange(batch.n_tokens) == 7, -1, batch.step_tokens).astype(np.int32))):
             with pytest.raises(B.ConfSpecError) as e:

@@ -63,8 +63,11 @@ def test_verify_select_append_verify():
     k = 2 + int(np.argmax(srt[3:nB - 1] - srt[2:nB - 2]))
     tau, gap = float(0.5 * (srt[k] + srt[k + 1])), float(srt[k + 1] - srt[k])
     ref1 = P.O.verify_cascade(wd, wt, spans1, lens1, lambda i, l: kvd[req_of[i]][l], lambda i, l: kvt[req_of[i]][l],
-                              vids, tau)
+                              vids, tau, req_offsets=REQ_OFFSETS, accept_index=0)
     esc = ref1["escalated"]
+    # linear drafting: steps behind a trusted rejection of their request are not sent to the target model
+    n_below = int((ref1["draft"]["accept"] == 0).sum())
+    assert 0 < esc.size < n_below
     vt, ct = np.full(nB, -1, np.int32), np.zeros(nB, np.float32)
     if esc.size:
         vt[esc], ct[esc] = ref1["target"]["verdict"], ref1["target"]["conf"]
@@ -92,24 +95,28 @@ def test_verify_select_append_verify():
         for mdl in (md, mt):
             B.cs_set_keep_logits(mdl, True)
 
-        def cascade(spans, tau_):
+        def cascade(spans, tau_, req_offsets=None):
             toks = np.concatenate(spans).astype(np.int32)
             lens = np.array([len(s) for s in spans], dtype=np.int32)
             n = B.cs_verify_cascade(md, kd, mt, kt, req_of, toks, lens, vids, tau_, conf_d, trusted, ver_d, conf_t,
-                                    ver_t, ver, conf)
+                                    ver_t, ver, conf, req_offsets=req_offsets, accept_index=0)
             torch.cuda.synchronize()
             B.cs_last_status(md), B.cs_last_status(mt)
             return n, toks, lens
 
-        n1, toks1, lens_1 = cascade(spans1, tau)
+        n1, toks1, lens_1 = cascade(spans1, tau, REQ_OFFSETS)
         assert np.max(np.abs(conf_d.cpu().numpy() - ref1["draft"]["conf"])) < 0.45 * gap
-        assert n1 == esc.size and np.array_equal(np.nonzero(trusted.cpu().numpy() == 0)[0], esc)
+        assert np.array_equal(trusted.cpu().numpy(), ref1["draft"]["accept"])
+        assert n1 == esc.size and np.array_equal(np.nonzero(ver_t.cpu().numpy() >= 0)[0], esc)
+        left_out = (trusted.cpu().numpy() == 0) & (ver_t.cpu().numpy() < 0)
+        assert left_out.sum() == n_below - esc.size
+        assert np.all(ver.cpu().numpy()[left_out] == -1) and np.all(conf.cpu().numpy()[left_out] == 0.0)
         m_dev, best = i32(R), i32(R)
         B.cs_cascade_select(trusted, ver_d, conf_d, ver_t, conf_t, torch.from_numpy(REQ_OFFSETS).to(dev), 0, m_dev, best)
         torch.cuda.synchronize()
         # the decisions may differ from the oracle's only where the two verdict probabilities are nearly equal
         pv_d = np.exp(ref1["draft"]["logits"][:, list(vids)] - ref1["draft"]["lse"][:, None])
-        clear = np.abs(pv_d[:, 0] - pv_d[:, 1]) > 0.03
+        clear = (np.abs(pv_d[:, 0] - pv_d[:, 1]) > 0.03) | (ref1["draft"]["accept"] == 0)   # only decisions that are used
         if esc.size:
             pv_t = np.exp(ref1["target"]["logits"][:, list(vids)] - ref1["target"]["lse"][:, None])
             clear[esc] = np.abs(pv_t[:, 0] - pv_t[:, 1]) > 0.03
