@@ -285,6 +285,18 @@ int cs_get_last_lse(cs_model* model, float* dev_out, int B, void* stream);
 int cs_last_status(cs_model* model, void* stream);
 
 /*
+ * cs_selftest_wait_timeout - failure detection, exercised without a fault: every wait inside the library's kernels
+ * (on a copy's arrival, on a tensor-core commit) is bounded; a kernel whose wait runs out raises a bit in the
+ * model's status word, stops issuing work, lets its copies land, frees its tensor memory and returns, and the next
+ * cs_last_status reports CS_ETIMEOUT. This call launches a one-thread kernel that runs that same bounded wait, with a
+ * limit of `polls` polls (1 .. 2^20; a few milliseconds at most), on a barrier nothing ever arrives at, so that the
+ * path from a starved wait to the host can be tested on a healthy GPU. The context stays usable.
+ * Returns CS_OK when the wait gave up as it should (the model's status word now holds the time-out bit: the next
+ * cs_last_status returns CS_ETIMEOUT and clears it), CS_ESTATE if the wait returned as satisfied. Synchronises `stream`.
+ */
+int cs_selftest_wait_timeout(cs_model* model, int polls, void* stream);
+
+/*
  * Per-stage entry points. They run single kernels of the pass on caller-provided device buffers so that
  * each can be checked against the oracle's corresponding block, and timed, in isolation.
  */

@@ -17,7 +17,7 @@ EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_reserve",
     "cs_kv_alloc", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
     "cs_verify_steps", "cs_verify_cascade", "cs_append_accepted", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
-    "cs_last_status", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
+    "cs_last_status", "cs_selftest_wait_timeout", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
 ]
 
 PROF_CLASSES = ["embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gateup", "gemm_down",
@@ -82,6 +82,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_get_last_logits": (C.c_int, [vp, vp, i32, vp]),
         "cs_get_last_lse": (C.c_int, [vp, vp, i32, vp]),
         "cs_last_status": (C.c_int, [vp, vp]),
+        "cs_selftest_wait_timeout": (C.c_int, [vp, i32, vp]),
         "cs_gemm_f16": (C.c_int, [vp, vp, vp, vp, i32, i32, i32, i32, vp]),
         "cs_rmsnorm": (C.c_int, [vp, vp, vp, i32, i32, f32, vp]),
         "cs_lm_head_gate": (C.c_int, [vp, vp, i32, i32, i32, vp, i32, f32, vp, vp, vp, vp, vp]),
@@ -308,6 +309,10 @@ def cs_get_last_lse(model: int, out, B: int, stream=None) -> None:
 
 def cs_last_status(model: int, stream=None) -> None:
     _check(load_library().cs_last_status(model, _stream_ptr(stream)), "cs_last_status")
+
+
+def cs_selftest_wait_timeout(model: int, polls: int = 4096, stream=None) -> None:
+    _check(load_library().cs_selftest_wait_timeout(model, int(polls), _stream_ptr(stream)), "cs_selftest_wait_timeout")
 
 
 def cs_gemm_f16(a, w, w2, out, M: int, N: int, K: int, epilogue: int, stream=None) -> None:

@@ -1032,6 +1032,20 @@ int cs_last_status(cs_model* m, void* stream) {
   return (v & 1u) ? CS_ETIMEOUT : CS_OK;
 }
 
+int cs_selftest_wait_timeout(cs_model* m, int polls, void* stream) {
+  if (!m || polls < 1 || polls > (1 << 20)) return CS_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc;
+  if ((rc = m->casc_idx.ensure(sizeof(int32_t) * 4))) return rc;
+  int32_t* gave_up = static_cast<int32_t*>(m->casc_idx.p);
+  CS_CUDA(cudaMemsetAsync(gave_up, 0, sizeof(int32_t), s));
+  CS_CUDA(launch_wait_timeout_selftest(m->status, static_cast<uint32_t>(polls), gave_up, s));
+  int32_t h = 0;
+  CS_CUDA(cudaMemcpyAsync(&h, gave_up, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  CS_CUDA(cudaStreamSynchronize(s));
+  return h == 1 ? CS_OK : CS_ESTATE;
+}
+
 int cs_profile(cs_model* m, int enable) {
   if (!m) return CS_EINVAL;
   m->prof.on = enable != 0;

@@ -133,7 +133,27 @@ __global__ void bf16_to_f16_kernel(uint32_t* __restrict__ p, size_t n_pairs) {
     p[i] = bf16x2_to_f16x2(p[i]);
 }
 
+// One thread waits, with the library's bounded wait, on a barrier of its own that nothing ever arrives at: the wait
+// runs out after `limit` polls, raises the time-out bit of the status word and the kernel returns normally.
+__global__ void wait_timeout_selftest_kernel(uint32_t* status, uint32_t limit, int32_t* gave_up) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_barrier_init();
+    const bool ok = mbar_wait_limited(&bar, 0, &abort_flag, status, limit);
+    *gave_up = ok ? 0 : 1;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_wait_timeout_selftest(uint32_t* status, uint32_t limit, int32_t* gave_up, cudaStream_t s) {
+  wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status, limit, gave_up);
+  count_launch();
+  return cudaGetLastError();
+}
 
 cudaError_t launch_bf16_to_f16(uint16_t* p, size_t n, cudaStream_t s) {
   if (n == 0) return cudaSuccess;

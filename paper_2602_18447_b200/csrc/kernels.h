@@ -101,6 +101,9 @@ cudaError_t launch_cascade_scatter(int B, const uint8_t* trusted, const int32_t*
                                    const float* conf_c, int32_t* out_verdict_t, float* out_conf_t,
                                    int32_t* out_verdict, float* out_conf, cudaStream_t s);
 
+// Failure-detection self-test: a bounded wait that is made to run out (see cs_selftest_wait_timeout).
+cudaError_t launch_wait_timeout_selftest(uint32_t* status, uint32_t limit, int32_t* gave_up, cudaStream_t s);
+
 // Launch with programmatic stream serialisation (see pdl_wait in common.cuh).
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
