@@ -19,7 +19,8 @@ the exactly widened bf16 weights and bf16 context K/V. No tiling, no online
 softmax, no split reductions: each function is the definition written out,
 with numpy matmul as the only library step.
 
-Parity pins (tests/test_oracle_*.py): closed forms for each block, brute-force
+Parity pins (tests/test_oracle_*.py): closed forms for each block, the 8-bit cache format's decoding against
+hand-decoded codes and a library's table, brute-force
 attention with scalar loops, cache-extend == full causal recompute, rotary
 shift invariance, GQA == MHA with repeated heads, softmax sums to one, gate
 end points of Table 3 (gamma = 0 never escalates, gamma > 1 always does),
@@ -55,6 +56,18 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
     r = u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))
     r &= np.uint32(0xFFFF0000)
     return r.view(np.float32).astype(np.float64)
+
+
+def widen_e4m3(codes: np.ndarray) -> np.ndarray:
+    """uint8 codes of the 8-bit float with 4 exponent bits (bias 7) and 3 mantissa bits, in the variant without
+    infinities (the optional 8-bit cache format) -> float64, exactly: sign s, exponent field e, mantissa field m
+    give (-1)^s 2^(e-7) (1 + m/8) for e >= 1, (-1)^s 2^-6 (m/8) for e = 0; e = 15 with m = 7 is NaN, so the
+    largest finite value is 448."""
+    c = np.ascontiguousarray(codes, dtype=np.uint8).astype(np.int64)
+    s, e, m = (c >> 7) & 1, (c >> 3) & 15, c & 7
+    mag = np.where(e == 0, np.ldexp(m / 8.0, -6), np.ldexp(1.0 + m / 8.0, e - 7))
+    mag = np.where((e == 15) & (m == 7), np.nan, mag)
+    return np.where(s == 1, -mag, mag)
 
 
 # ----------------------------------------------------------------------------------------------

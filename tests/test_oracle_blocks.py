@@ -252,3 +252,18 @@ def test_cascade_select_hand_worked_iterations():
     # without target results every escalated step is a rejection
     p2, _, m2, _ = O.cascade_select(trusted, vd, cd, None, None, offs)
     assert all(p2[i] == 0 for i in range(len(trusted)) if not trusted[i]) and np.all(m2 <= m)
+
+
+def test_e4m3_decode_against_hand_values_and_a_library():
+    """The 8-bit cache format: hand-decoded codes, order, and every code against torch's float8_e4m3fn."""
+    hand = {0x00: 0.0, 0x01: 2.0 ** -9, 0x07: 7 * 2.0 ** -9, 0x08: 2.0 ** -6, 0x38: 1.0, 0x3C: 1.5, 0x40: 2.0,
+            0x7E: 448.0, 0xB8: -1.0, 0xFE: -448.0, 0x30: 0.5, 0x39: 1.125}
+    for code, want in hand.items():
+        assert O.widen_e4m3(np.array([code], np.uint8))[0] == want, hex(code)
+    assert np.isnan(O.widen_e4m3(np.array([0x7F, 0xFF], np.uint8))).all()
+    pos = O.widen_e4m3(np.arange(0x7F, dtype=np.uint8))
+    assert np.all(np.diff(pos) > 0)
+    torch = pytest.importorskip("torch")
+    lib = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    ours = O.widen_e4m3(np.arange(256, dtype=np.uint8))
+    assert np.array_equal(np.isnan(lib), np.isnan(ours)) and np.array_equal(lib[~np.isnan(lib)], ours[~np.isnan(ours)])

@@ -2,6 +2,7 @@
 import os
 
 import numpy as np
+import pytest
 
 from oracle import confspec_oracle as O
 from workloads import CONFIGS, context_kv, get_config, make_batch, model_weights, page_assignment, scaled_config
@@ -58,3 +59,18 @@ def test_context_kv_and_pages():
     assert len(set(allp.tolist())) == allp.shape[0] and allp.max() < total
     assert [len(p) for p in pages] == [(int(c) + 15) // 16 for c in b.ctx_lens]
     assert not np.array_equal(pages[0], np.sort(pages[0]))          # scattered, not contiguous
+
+
+def test_e4m3_encoding_rounds_to_nearest_even_and_saturates():
+    from workloads import e4m3_codes_from_f32
+    torch = pytest.importorskip("torch")
+    g = np.random.default_rng(0)
+    x = np.concatenate([g.standard_normal(20000) * 0.78, g.standard_normal(2000) * 100, [0.0, -0.0, 448.0, 449.0, -1e9,
+                        2.0 ** -10, 3 * 2.0 ** -10, 1.0625, 1.1875, 2.0 ** -9, 1e-12]]).astype(np.float32)
+    ours = e4m3_codes_from_f32(x)
+    lib = torch.from_numpy(x).clamp(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    same = ours == lib
+    zero = (ours & 0x7F) == 0                      # the sign of a zero result is storage detail
+    assert np.all(same | (zero & ((lib & 0x7F) == 0)))
+    # ties go to the even code: 1.0625 is halfway between 1.0 (0x38) and 1.125 (0x39); 1.1875 between 0x39 and 0x3A
+    assert e4m3_codes_from_f32(np.array([1.0625, 1.1875, 449.0, 1e9], np.float32)).tolist() == [0x38, 0x3A, 0x7E, 0x7E]

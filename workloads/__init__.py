@@ -9,6 +9,7 @@ from .configs import (ModelShape, VerifyConfig, CascadeConfig, CONFIGS, CASCADES
                       scaled_config)
 from .generate import (
     bf16_bits_from_f32,
+    e4m3_codes_from_f32,
     model_weights,
     plant_verdict_rows,
     make_batch,
@@ -20,6 +21,6 @@ from .generate import (
 __all__ = [
     "ModelShape", "VerifyConfig", "CascadeConfig", "CONFIGS", "CASCADES", "get_config", "get_cascade",
     "scaled_config",
-    "bf16_bits_from_f32", "model_weights", "plant_verdict_rows", "make_batch",
+    "bf16_bits_from_f32", "e4m3_codes_from_f32", "model_weights", "plant_verdict_rows", "make_batch",
     "context_kv", "page_assignment", "Batch",
 ]

@@ -72,6 +72,8 @@ class VerifyConfig:
     # "synthetic": context K/V are drawn i.i.d. N(0, kv_std^2), rounded to bf16, K taken as already rotated.
     ctx_kv: str = "synthetic"
     kv_std: float = 0.78
+    # cache format: "bf16", or "e4m3" (8-bit float, 4 exponent / 3 mantissa bits, unscaled; synthetic contexts only)
+    kv_format: str = "bf16"
     seed: int = 20260218
 
 
@@ -94,6 +96,9 @@ CONFIGS = {
     # bound by reading the cache rather than by arithmetic
     "cfg7_q3_short": VerifyConfig(
         "cfg7_q3_short", QWEN3_1P7B, 64, ("uniform", 2048, 8192), ("uniform", 1, 4), suffix_len=4, tau=0.9, seed=707),
+    "cfg9_q3_short_fp8": VerifyConfig(
+        "cfg9_q3_short_fp8", QWEN3_1P7B, 64, ("uniform", 2048, 8192), ("uniform", 1, 4), suffix_len=4, tau=0.9, seed=707,
+        kv_format="e4m3"),
     "cfg8_tiny_qknorm": VerifyConfig(
         "cfg8_tiny_qknorm", TINY_QKNORM, 6, ("uniform", 20, 150), ("uniform", 1, 40), tau=0.8, ctx_kv="prefill",
         seed=808),

@@ -37,6 +37,28 @@ def bf16_bits_from_f32(x: np.ndarray) -> np.ndarray:
     return (r >> np.uint32(16)).astype(np.uint16)
 
 
+def _e4m3_positive_values() -> np.ndarray:
+    """The 127 non-negative finite values of the 8-bit float with 4 exponent bits (bias 7), 3 mantissa bits and no
+    infinities, in code order 0x00 .. 0x7E (which is also increasing order)."""
+    c = np.arange(127)
+    e, m = c >> 3, c & 7
+    return np.where(e == 0, np.ldexp(m / 8.0, -6), np.ldexp(1.0 + m / 8.0, e - 7))
+
+
+def e4m3_codes_from_f32(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest value of that 8-bit format (ties to the even code, magnitudes beyond 448 saturate) and
+    return the codes as uint8. Storage conversion only."""
+    vals = _e4m3_positive_values()
+    a = np.abs(np.ascontiguousarray(x, dtype=np.float64))
+    hi = np.clip(np.searchsorted(vals, a, side="left"), 1, 126)       # vals[hi-1] <= a <= vals[hi] (or a beyond the end)
+    lo = hi - 1
+    d_lo, d_hi = a - vals[lo], vals[hi] - a
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
+    code = np.where(pick_hi, hi, lo)
+    code = np.where(a >= vals[126], 126, code).astype(np.uint8)
+    return np.where(np.signbit(x), code | np.uint8(0x80), code).astype(np.uint8)
+
+
 def _normal_bf16(key: Tuple[int, ...], shape: Tuple[int, ...], std: float,
                  pool: Optional[ThreadPoolExecutor] = None) -> np.ndarray:
     """i.i.d. N(0, std^2) rounded to bf16; drawn in fixed row chunks with one stream per chunk."""
@@ -167,13 +189,17 @@ def make_batch(cfg: VerifyConfig, seed: Optional[int] = None) -> Batch:
 
 def context_kv(cfg: VerifyConfig, step: int, layer: int, ctx_len: int,
                seed: Optional[int] = None) -> Tuple[np.ndarray, np.ndarray]:
-    """Synthetic cached K and V of one step for one layer: uint16 bf16 bits, each [ctx_len, n_kv_heads,
-    head_dim], i.i.d. N(0, kv_std^2). K is taken as already rotated."""
+    """Synthetic cached K and V of one step for one layer: uint16 bf16 bits (uint8 codes of the 8-bit format when
+    cfg.kv_format == "e4m3": the same draws, rounded once more), each [ctx_len, n_kv_heads, head_dim],
+    i.i.d. N(0, kv_std^2). K is taken as already rotated."""
     seed = cfg.seed if seed is None else seed
     m = cfg.model
     shape = (int(ctx_len), m.n_kv_heads, m.head_dim)
     k = _normal_bf16((seed, _TAG_CTXKV, step, layer, 0), shape, cfg.kv_std)
     v = _normal_bf16((seed, _TAG_CTXKV, step, layer, 1), shape, cfg.kv_std)
+    if cfg.kv_format == "e4m3":
+        widen = lambda b: (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+        return e4m3_codes_from_f32(widen(k)), e4m3_codes_from_f32(widen(v))
     return k, v
 
 
