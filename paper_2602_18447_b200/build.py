@@ -8,7 +8,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libconfspec.so")
-SOURCES = ["api.cu", "gemm_tcgen05.cu", "attention.cu", "lmhead.cu", "elementwise.cu"]
+SOURCES = ["api.cu", "gemm_tcgen05.cu", "attention.cu", "attention_short.cu", "lmhead.cu", "elementwise.cu"]
 HEADERS = ["common.cuh", "gemm.h", "kernels.h", os.path.join("..", "..", "include", "confspec.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]

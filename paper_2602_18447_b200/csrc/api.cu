@@ -111,8 +111,9 @@ struct cs_model {
 struct cs_kv {
   const cs_model* model;
   int num_pages, page_size, max_seqs, max_pages_per_seq;
-  uint16_t* pool = nullptr;
+  uint16_t* pool = nullptr;   // 16-bit cells (bf16 values in the fp16 encoding), or 8-bit codes when format == 1
   bool own_pool = false;
+  int format = 0;             // 0: 16-bit cells; 1: 8-bit float, 4 exponent / 3 mantissa bits (read-only for the pass)
   size_t plane_elems;  // elements of one (layer, K or V) plane
   CUtensorMap tm_pool;
   int32_t* table_host = nullptr;  // pinned [max_seqs, max_pages_per_seq]
@@ -173,6 +174,8 @@ struct BatchLayout {
   int B = 0, T = 0;
   size_t off_cu, off_pos, off_tseq, off_tok, off_items, total;
   int n_items = 0, n_slots = 0;
+  int max_rows = 0;        // 8-bit cache: the largest number of query rows (new tokens x heads per kv head) of a step
+  bool any_split = false;  // 8-bit cache: some context is cut into pieces
 };
 
 // Cost of an attention work item in key tiles: the tiles themselves plus the fixed part of a CTA (set-up, Q load,
@@ -273,6 +276,36 @@ void build_attention_work(const cs_model* m, int B, const int32_t* lens, const i
       }
       if (n > 1) slots += n;
     }
+  std::stable_sort(items.begin(), items.end(), [](const AttnItem& a, const AttnItem& b) {
+    return (a.tile_end - a.tile_begin) > (b.tile_end - b.tile_begin);
+  });
+  *n_slots = slots;
+}
+
+// Work items of the short-step attention over an 8-bit cache: one per (step, kv head, piece of the context's pages).
+// The pieces are sized so that the launch has a few CTAs per SM; the last piece of a step also covers its own keys.
+void build_short_work(const cs_model* m, int B, const int32_t* lens, const int32_t* ctx, std::vector<AttnItem>& items,
+                      int* n_slots, bool* any_split) {
+  const int heads = m->d.n_kv_heads;
+  long units = 0;
+  for (int i = 0; i < B; ++i) units += static_cast<long>((ctx[i] + kPageSize - 1) / kPageSize) * heads;
+  const long chunk = std::max<long>(32, units / (kNumSMs * 6L) + 1);
+  items.clear();
+  int slots = 0;
+  *any_split = false;
+  for (int i = 0; i < B; ++i) {
+    const int pages = (ctx[i] + kPageSize - 1) / kPageSize;
+    const int n = static_cast<int>(std::min<long>(32, std::max<long>(1, (pages + chunk - 1) / chunk)));
+    for (int h = 0; h < heads; ++h) {
+      for (int s = 0; s < n; ++s) {
+        const int b = static_cast<int>(static_cast<long>(pages) * s / n);
+        const int e = static_cast<int>(static_cast<long>(pages) * (s + 1) / n);
+        items.push_back(AttnItem{i, h, 0, b, e, n > 1 ? slots + s : 0, n > 1 ? slots : 0, n, 0, lens[i], ctx[i], 0,
+                                 {0, 0, 0, 0}});
+      }
+      if (n > 1) { slots += n; *any_split = true; }
+    }
+  }
   std::stable_sort(items.begin(), items.end(), [](const AttnItem& a, const AttnItem& b) {
     return (a.tile_end - a.tile_begin) > (b.tile_end - b.tile_begin);
   });
@@ -386,7 +419,14 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
     CS_STEP(kProfQkv, gemm_f16_rope(tm_a, lw.tm_wqkv, qkv, T, m->n_qkv, d.d_model, rope_epi, m->status, s));
     ap.k_group_base = (2 * l) * plane_groups;
     ap.v_group_base = (2 * l + 1) * plane_groups;
-    CS_STEP(kProfAttn, launch_attention(ap, kv->tm_pool, tm_qkv_attn, tm_q3d, d_items, L.n_items, s));
+    if (kv->format == 1) {
+      const uint8_t* pool8 = reinterpret_cast<const uint8_t*>(kv->pool);
+      CS_STEP(kProfAttn, launch_attention_short(ap, pool8 + static_cast<size_t>(2 * l) * kv->plane_elems,
+                                                pool8 + static_cast<size_t>(2 * l + 1) * kv->plane_elems, d_items,
+                                                L.n_items, L.max_rows, L.any_split, s));
+    } else {
+      CS_STEP(kProfAttn, launch_attention(ap, kv->tm_pool, tm_qkv_attn, tm_q3d, d_items, L.n_items, s));
+    }
     if (append_kv) {
       CS_STEP(kProfOther, launch_kv_scatter(qkv + m->q_dim, qkv + m->q_dim + m->kv_dim, m->n_qkv, d_tseq, d_pos, 0, 0,
                                 append_kv->table_dev, append_kv->max_pages_per_seq,
@@ -442,8 +482,16 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   std::vector<int32_t> ctx(B);
   for (int i = 0; i < B; ++i) ctx[i] = kv->ctx_len[seq_ids[i]];
   std::vector<AttnItem> items;
-  int n_slots = 0;
-  build_attention_work(m, B, lens, ctx.data(), items, &n_slots);
+  int n_slots = 0, max_rows = 0;
+  bool any_split = false;
+  if (kv->format == 1) {
+    const int G = m->d.n_q_heads / m->d.n_kv_heads;
+    for (int i = 0; i < B; ++i) max_rows = std::max(max_rows, lens[i] * G);
+    if (max_rows > 32) return CS_EINVAL;     // the 8-bit cache serves short steps only
+    build_short_work(m, B, lens, ctx.data(), items, &n_slots, &any_split);
+  } else {
+    build_attention_work(m, B, lens, ctx.data(), items, &n_slots);
+  }
 
   BatchLayout L;
   L.B = B;
@@ -458,6 +506,8 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   L.total = o;
   L.n_items = static_cast<int>(items.size());
   L.n_slots = n_slots;
+  L.max_rows = max_rows;
+  L.any_split = any_split;
 
   int rc;
   if ((rc = ensure_workspace(m, B, L.T))) return rc;
@@ -668,8 +718,21 @@ uint64_t cs_kv_pool_bytes(const cs_model* m, int num_pages, int page_size) {
   return static_cast<uint64_t>(m->d.n_layers) * 2 * num_pages * m->d.n_kv_heads * page_size * m->d.head_dim * 2;
 }
 
+static int kv_alloc_impl(const cs_model* m, int num_pages, int page_size, int max_seqs, int max_pages_per_seq,
+                         void* dev_pool, int format, cs_kv** out);
+
 int cs_kv_alloc(const cs_model* m, int num_pages, int page_size, int max_seqs, int max_pages_per_seq, void* dev_pool,
                 cs_kv** out) {
+  return kv_alloc_impl(m, num_pages, page_size, max_seqs, max_pages_per_seq, dev_pool, 0, out);
+}
+
+int cs_kv_alloc_e4m3(const cs_model* m, int num_pages, int page_size, int max_seqs, int max_pages_per_seq,
+                     cs_kv** out) {
+  return kv_alloc_impl(m, num_pages, page_size, max_seqs, max_pages_per_seq, nullptr, 1, out);
+}
+
+static int kv_alloc_impl(const cs_model* m, int num_pages, int page_size, int max_seqs, int max_pages_per_seq,
+                         void* dev_pool, int format, cs_kv** out) {
   if (!out) return CS_EINVAL;
   *out = nullptr;
   if (!m || num_pages < 1 || page_size != kPageSize || max_seqs < 1 || max_pages_per_seq < 1) return CS_EINVAL;
@@ -679,6 +742,7 @@ int cs_kv_alloc(const cs_model* m, int num_pages, int page_size, int max_seqs, i
   cs_kv* kv = new (std::nothrow) cs_kv();
   if (!kv) return CS_ENOMEM;
   kv->model = m;
+  kv->format = format;
   kv->num_pages = num_pages;
   kv->page_size = page_size;
   kv->max_seqs = max_seqs;
@@ -686,7 +750,7 @@ int cs_kv_alloc(const cs_model* m, int num_pages, int page_size, int max_seqs, i
   kv->plane_elems = static_cast<size_t>(num_pages) * m->d.n_kv_heads * page_size * m->d.head_dim;
   kv->ctx_len.assign(max_seqs, -1);
   kv->n_pages.assign(max_seqs, 0);
-  const uint64_t bytes = cs_kv_pool_bytes(m, num_pages, page_size);
+  const uint64_t bytes = cs_kv_pool_bytes(m, num_pages, page_size) / (format == 1 ? 2 : 1);
   int rc = CS_OK;
   cudaError_t e;
   if (dev_pool) {
@@ -707,7 +771,7 @@ int cs_kv_alloc(const cs_model* m, int num_pages, int page_size, int max_seqs, i
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&kv->upload_ev, cudaEventDisableTiming);
   if (e != cudaSuccess) { rc = cuda_fail(e, "kv page table"); cs_kv_free(kv); return rc; }
   std::memset(kv->table_host, 0, tbytes);
-  if (!make_kv_group_map(&kv->tm_pool, kv->pool, rows, m->d.head_dim, kPageSize / 8)) {
+  if (format == 0 && !make_kv_group_map(&kv->tm_pool, kv->pool, rows, m->d.head_dim, kPageSize / 8)) {
     g_cuda_error = "cuTensorMapEncodeTiled failed for the kv pool";
     cs_kv_free(kv);
     return CS_ECUDA;
@@ -759,6 +823,19 @@ int cs_kv_fill(cs_kv* kv, int seq, int layer, const uint16_t* host_k, const uint
   int rc;
   if ((rc = kv->fill_tmp.ensure(2 * elems * 2))) return rc;
   if ((rc = upload_table(kv, s))) return rc;
+  if (kv->format == 1) {   // 8-bit cache: host_k / host_v hold one code per element
+    uint8_t* tk8 = static_cast<uint8_t*>(kv->fill_tmp.p);
+    uint8_t* tv8 = tk8 + elems;
+    uint8_t* pool8 = reinterpret_cast<uint8_t*>(kv->pool);
+    CS_CUDA(cudaMemcpyAsync(tk8, host_k, elems, cudaMemcpyHostToDevice, s));
+    CS_CUDA(cudaMemcpyAsync(tv8, host_v, elems, cudaMemcpyHostToDevice, s));
+    CS_CUDA(launch_kv_scatter_u8(tk8, tv8, seq, kv->table_dev, kv->max_pages_per_seq,
+                                 pool8 + static_cast<size_t>(2 * layer) * kv->plane_elems,
+                                 pool8 + static_cast<size_t>(2 * layer + 1) * kv->plane_elems, d.n_kv_heads, d.head_dim,
+                                 kPageSize, c, s));
+    CS_CUDA(cudaStreamSynchronize(s));
+    return CS_OK;
+  }
   uint16_t* tk = static_cast<uint16_t*>(kv->fill_tmp.p);
   uint16_t* tv = tk + elems;
   CS_CUDA(cudaMemcpyAsync(tk, host_k, elems * 2, cudaMemcpyHostToDevice, s));
@@ -774,6 +851,7 @@ int cs_kv_fill(cs_kv* kv, int seq, int layer, const uint16_t* host_k, const uint
 int cs_prefill(cs_model* m, cs_kv* kv, const int32_t* seq_ids, const int32_t* tokens, const int32_t* lens, int B,
                void* stream) {
   if (!m || !kv || kv->model != m || B < 0) return CS_EINVAL;
+  if (kv->format != 0) return CS_EINVAL;   // the 8-bit cache is filled with given codes, not appended to
   if (B == 0) return CS_OK;
   if (!seq_ids || !tokens || !lens) return CS_EINVAL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -797,7 +875,7 @@ int cs_prefill(cs_model* m, cs_kv* kv, const int32_t* seq_ids, const int32_t* to
 int cs_append_accepted(cs_model* m, cs_kv* kv, int R, const int32_t* req_seq_ids, const int32_t* req_offsets,
                        const int32_t* dev_prefix_len, const int32_t* step_tokens, const int32_t* step_lens,
                        const int32_t* draft_lens, int32_t* host_prefix_len, void* stream) {
-  if (!m || !kv || kv->model != m || R < 0) return CS_EINVAL;
+  if (!m || !kv || kv->model != m || R < 0 || kv->format != 0) return CS_EINVAL;
   if (R == 0) return CS_OK;
   if (!req_seq_ids || !req_offsets || !dev_prefix_len || !step_tokens || !step_lens || !draft_lens) return CS_EINVAL;
   if (req_offsets[0] != 0) return CS_EINVAL;

@@ -125,6 +125,25 @@ __global__ void kv_scatter_kernel(const uint16_t* __restrict__ src_k, const uint
   *reinterpret_cast<uint4*>(pool_v + dst) = v;
 }
 
+__global__ void kv_scatter_u8_kernel(const uint8_t* __restrict__ src_k, const uint8_t* __restrict__ src_v, int seq,
+                                     const int32_t* __restrict__ page_table, int max_pages_per_seq,
+                                     uint8_t* __restrict__ pool_k, uint8_t* __restrict__ pool_v, int n_kv_heads, int hd,
+                                     int page_size, int T) {
+  const int chunks = n_kv_heads * hd / 16;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= T * chunks) return;
+  const int t = i / chunks;
+  const int c = i - t * chunks;
+  const int head = (c * 16) / hd;
+  const int e = c * 16 - head * hd;
+  const int page = page_table[static_cast<size_t>(seq) * max_pages_per_seq + t / page_size];
+  const int slot = t % page_size;
+  const size_t dst = ((static_cast<size_t>(page) * n_kv_heads + head) * page_size + slot) * hd + e;
+  const size_t src = static_cast<size_t>(t) * n_kv_heads * hd + c * 16;
+  *reinterpret_cast<uint4*>(pool_k + dst) = *reinterpret_cast<const uint4*>(src_k + src);
+  *reinterpret_cast<uint4*>(pool_v + dst) = *reinterpret_cast<const uint4*>(src_v + src);
+}
+
 // In-place re-encoding of bf16 bit patterns as fp16 (same size). Exact for magnitudes in [2^-14, 65504];
 // smaller values round to the fp16 subnormal grid (absolute error <= 2^-25).
 __global__ void bf16_to_f16_kernel(uint32_t* __restrict__ p, size_t n_pairs) {
@@ -204,6 +223,17 @@ cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int 
   kv_scatter_kernel<<<(n + 255) / 256, 256, 0, s>>>(src_k, src_v, row_stride, tok_seq, tok_pos, const_seq, pos0, page_table,
                                                     max_pages_per_seq, pool_k_plane, pool_v_plane, n_kv_heads, hd,
                                                     page_size, T, src_is_f16);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_kv_scatter_u8(const uint8_t* src_k, const uint8_t* src_v, int seq, const int32_t* page_table,
+                                 int max_pages_per_seq, uint8_t* pool_k_plane, uint8_t* pool_v_plane, int n_kv_heads,
+                                 int hd, int page_size, int T, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  const int n = T * n_kv_heads * hd / 16;
+  kv_scatter_u8_kernel<<<(n + 255) / 256, 256, 0, s>>>(src_k, src_v, seq, page_table, max_pages_per_seq, pool_k_plane,
+                                                       pool_v_plane, n_kv_heads, hd, page_size, T);
   count_launch();
   return cudaGetLastError();
 }

@@ -38,7 +38,10 @@ class VerifySession:
                     room_for_prefill: bool = False) -> None:
         ps = self.cfg.page_size
         max_pp = max(1, max(len(p) for p in pages_per_step))
-        self.kv = B.cs_kv_alloc(self.model, total_pages, ps, self.n_steps, max_pp)
+        if getattr(self.cfg, "kv_format", "bf16") == "e4m3":
+            self.kv = B.cs_kv_alloc_e4m3(self.model, total_pages, ps, self.n_steps, max_pp)
+        else:
+            self.kv = B.cs_kv_alloc(self.model, total_pages, ps, self.n_steps, max_pp)
         for i, pages in enumerate(pages_per_step):
             B.cs_kv_set_seq(self.kv, i, pages, 0 if room_for_prefill else int(ctx_lens[i]))
 
