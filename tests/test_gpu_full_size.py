@@ -122,3 +122,12 @@ def test_cfg7_short_steps_on_long_contexts_full_depth(weights_q3):
     cfg, ses, gpu, ref, stats = _run_full("cfg7_q3_short", weights_q3, sample=[0, 33, 63])
     ses.close()
     assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
+
+
+def test_cfg9_short_steps_8bit_cache_full_depth(weights_q3):
+    """The decode-shaped batch over the 8-bit cache (same draws as cfg7, rounded to 8 bits), all 28 layers."""
+    cfg9 = get_config("cfg9_q3_short_fp8")
+    weights = weights_q3 if cfg9.seed == get_config("cfg6_q3_b16").seed else model_weights(cfg9.model, cfg9.seed)
+    cfg, ses, gpu, ref, stats = _run_full("cfg9_q3_short_fp8", weights, sample=[0, 33, 63])
+    ses.close()
+    assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL

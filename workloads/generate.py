@@ -37,26 +37,25 @@ def bf16_bits_from_f32(x: np.ndarray) -> np.ndarray:
     return (r >> np.uint32(16)).astype(np.uint16)
 
 
-def _e4m3_positive_values() -> np.ndarray:
-    """The 127 non-negative finite values of the 8-bit float with 4 exponent bits (bias 7), 3 mantissa bits and no
-    infinities, in code order 0x00 .. 0x7E (which is also increasing order)."""
-    c = np.arange(127)
-    e, m = c >> 3, c & 7
-    return np.where(e == 0, np.ldexp(m / 8.0, -6), np.ldexp(1.0 + m / 8.0, e - 7))
-
-
 def e4m3_codes_from_f32(x: np.ndarray) -> np.ndarray:
-    """Round to the nearest value of that 8-bit format (ties to the even code, magnitudes beyond 448 saturate) and
-    return the codes as uint8. Storage conversion only."""
-    vals = _e4m3_positive_values()
-    a = np.abs(np.ascontiguousarray(x, dtype=np.float64))
-    hi = np.clip(np.searchsorted(vals, a, side="left"), 1, 126)       # vals[hi-1] <= a <= vals[hi] (or a beyond the end)
-    lo = hi - 1
-    d_lo, d_hi = a - vals[lo], vals[hi] - a
-    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
-    code = np.where(pick_hi, hi, lo)
-    code = np.where(a >= vals[126], 126, code).astype(np.uint8)
-    return np.where(np.signbit(x), code | np.uint8(0x80), code).astype(np.uint8)
+    """Round to the nearest value of the 8-bit float with 4 exponent bits (bias 7), 3 mantissa bits and no infinities
+    (ties to the even code, magnitudes beyond 448 saturate) and return the codes as uint8. Storage conversion only.
+    Below 2^-6 the format is a fixed-point grid of step 2^-9 (codes 0 .. 8, code 8 being the smallest normal);
+    above, the fp32 mantissa is rounded to 3 bits in place and the exponent re-biased."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32)
+    sign = ((u >> np.uint32(24)) & np.uint32(0x80)).astype(np.uint8)
+    au = u & np.uint32(0x7FFFFFFF)
+    r = au + np.uint32(0x7FFFF)
+    r += (au >> np.uint32(20)) & np.uint32(1)
+    r >>= np.uint32(20)                                   # (fp32 exponent field << 3) | 3 mantissa bits
+    np.minimum(r, np.uint32(((127 - 7) << 3) + 0x7E), out=r)
+    code = r.astype(np.int32) - np.int32((127 - 7) << 3)
+    a = au.view(np.float32)
+    small = a < np.float32(2.0 ** -6)
+    if small.any():
+        code[small] = np.rint(a[small] * np.float32(512.0)).astype(np.int32)      # rint rounds ties to even
+    return code.astype(np.uint8) | sign
 
 
 def _normal_bf16(key: Tuple[int, ...], shape: Tuple[int, ...], std: float,
