@@ -117,7 +117,8 @@ int cs_kv_alloc(const cs_model* model, int num_pages, int page_size, int max_seq
 /*
  * cs_kv_alloc_e4m3 - the same cache in the optional 8-bit format (no counterpart in the paper, which leaves the
  * cache to its serving engine): one byte per element, the float with 4 exponent bits (bias 7), 3 mantissa bits and
- * no infinities, unscaled; same pool layout, half the bytes, always library-owned (cs_kv_pool_bytes() / 2).
+ * no infinities, unscaled; half the bytes, always library-owned (cs_kv_pool_bytes() / 2); pool layout as above
+ * except that V pages are kept transposed, [head_dim][page_size].
  * It serves the decode-shaped use of the pass, where reading the cache bounds the time: cs_verify_steps accepts it
  * when every step has at most 32 query rows per kv head (step_lens[i] * n_q_heads / n_kv_heads <= 32; CS_EINVAL
  * otherwise), widens the codes to fp16 on the fly (exact) and computes as with the 16-bit cache. The format is

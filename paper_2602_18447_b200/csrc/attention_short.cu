@@ -1,10 +1,12 @@
 // Extend-attention for short steps (at most 32 query rows per kv head: new tokens x heads in the group) over a cache
 // kept in the 8-bit format. With so few rows the pass is bound by reading the cache, not by arithmetic, so the
 // kernel is organised around bytes: every warp streams whole 16-key pages of one (step, kv head) from global memory
-// with asynchronous copies, two pages in flight, widens them to fp16 in shared memory (exact: every 8-bit value is an
-// fp16 value) and runs the two small products of the page on warp-level tensor-core instructions. There is no wait on
+// with asynchronous copies, three pages in flight, widens the codes to fp16 in registers (exact: every 8-bit value is
+// an fp16 value) and runs the two small products of the page on warp-level tensor-core instructions. There is no wait on
 // another CTA and no spin: pieces of a long context leave partial results that a second kernel combines.
 #include <cuda_fp16.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 #include "kernels.h"
@@ -26,16 +28,6 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(addr));
-}
 // D (16 x 8, fp32) += A (16 x 16, fp16, row) * B (16 x 8, fp16, col)
 __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -54,24 +46,32 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// Shared memory of one warp: two raw pages in flight (K and V codes), and the current page widened to fp16 in
-// rows of HD halves whose 16-byte chunks are XOR-swizzled with the row, which keeps ldmatrix free of bank conflicts.
-template <int HD>
-struct WarpSmem {
-  static constexpr int kRawPage = kPage * HD;          // bytes of one K or V page of one head, 8-bit
-  static constexpr int kWidePage = kPage * HD * 2;     // the same as fp16
-  static constexpr int kBytes = 2 * 2 * kRawPage + 2 * kWidePage;
-};
+// Fragments are built straight from the codes, without a pass through shared memory in fp16:
+//  - K page [16 keys][HD codes]. The score product sums over the head dimension, in any order, so the dimension
+//    index is permuted to make every lane's operands contiguous: in each block of 32 dimensions lane q = lane % 4 owns
+//    dimensions 8q .. 8q+7 (one 8-byte load = the B operands of two k-steps), and the query fragments use the same
+//    permutation. The 16 keys are likewise assigned to the columns of the two 8-column score tiles so that lane q ends
+//    up holding the probabilities of keys 4q .. 4q+3: tile 0 column c is key 4 (c / 2) + c % 2, tile 1 that plus 2.
+//  - V page TRANSPOSED, [HD][16 keys codes] (the layout of the 8-bit pool's V planes): the B operand of
+//    O += P V for output column d and keys 4q .. 4q+3 is one 4-byte load.
+// Shared memory of one warp: kStagesS pages in flight (K codes, 16-byte chunks XOR-swizzled per key row; V^T codes).
+constexpr int kStagesS = 4;
 template <int HD>
 struct ShortSmem {
+  static constexpr int kRawPage = kPage * HD;                  // bytes of one K or V page of one head
+  static constexpr int kStage = 2 * kRawPage;
+  static constexpr int kWarp = kStagesS * kStage;
   static constexpr int kQBytes = 32 * HD * 2;
-  static constexpr int kWarp = WarpSmem<HD>::kBytes;
   static constexpr int kTotal = kQBytes + kShortWarps * kWarp;
-  // the combining step reuses the warps' buffers: [warp][32 rows][HD] fp32 + [warp][32][2]
-  static_assert(kShortWarps * kWarp >= kShortWarps * 16 * HD * 4, "partial results of one row tile must fit");
+  // reused after the loop: the step's own keys in fp16 (K [16][HD], V^T [HD][16]) in warp 0's stages, and the
+  // warps' partial results [warp][32 rows][HD] fp32
+  static_assert(kWarp >= 2 * kPage * HD * 2, "own keys must fit in one warp's stages");
+  static_assert(kShortWarps * kWarp >= kShortWarps * 32 * HD * 4, "partial results must fit");
 };
 
-__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (static_cast<uint32_t>(chunk) ^ (row & 7)) << 4; }
+// swizzle of the 16-byte chunks of a K row: distinct for the 8 keys one score tile reads at once
+template <int HD>
+__device__ __forceinline__ int k_swz(int key) { return (((key >> 2) << 1) | (key & 1)) & (HD / 16 - 1); }
 
 // MT = number of 16-row tiles of query rows (1 or 2).
 template <int HD, int MT>
@@ -80,65 +80,70 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
                        const AttnItem* __restrict__ items) {
   constexpr int KS = HD / 16;        // k-steps of the score product
   constexpr int NT = HD / 8;         // 8-column tiles of the output
-  constexpr int RAW = WarpSmem<HD>::kRawPage;
-  constexpr int WIDE = WarpSmem<HD>::kWidePage;
-  constexpr int ROWB = HD * 2;       // bytes of one fp16 row
+  constexpr int RAW = ShortSmem<HD>::kRawPage;
+  constexpr int STAGE = ShortSmem<HD>::kStage;
   extern __shared__ __align__(128) uint8_t smem[];
   pdl_launch_dependents();
   const AttnItem it = items[blockIdx.x];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, q = lane & 3;
   const int G = p.n_q_heads / p.n_kv_heads;
   const int R = it.n_new * G;                       // query rows in use (<= 16 MT)
   uint8_t* q_s = smem;
   uint8_t* my = smem + ShortSmem<HD>::kQBytes + warp * ShortSmem<HD>::kWarp;
-  auto raw_of = [&](int stage) { return my + stage * 2 * RAW; };   // each stage: K codes then V codes
-  uint8_t* k_w = my + 4 * RAW;
-  uint8_t* v_w = k_w + WIDE;
   const int32_t* table = p.page_table + static_cast<size_t>(it.seq) * p.max_pages_per_seq;
   const size_t head_off = static_cast<size_t>(it.kv_head) * kPage * HD;
   const size_t page_stride = static_cast<size_t>(p.n_kv_heads) * kPage * HD;
 
   // cached pages of this warp: page_begin + warp, + 4, ...; the copies touch only the cache and the page table, which
-  // no kernel of the pass writes, so the first two go out before the wait on the previous kernel
+  // no kernel of the pass writes, so the first ones go out before the wait on the previous kernel
   auto fetch = [&](int pg, int stage) {
     const int32_t id = __ldg(table + pg);
     const uint8_t* gk = pool_k + static_cast<size_t>(id) * page_stride + head_off;
     const uint8_t* gv = pool_v + static_cast<size_t>(id) * page_stride + head_off;
+    uint8_t* dst = my + stage * STAGE;
     for (int c = lane; c < RAW / 16; c += 32) {
-      cp_async_16(raw_of(stage) + c * 16, gk + c * 16);
-      cp_async_16(raw_of(stage) + RAW + c * 16, gv + c * 16);
+      const int key = c / (HD / 16), ch = c % (HD / 16);
+      cp_async_16(dst + key * HD + ((ch ^ k_swz<HD>(key)) << 4), gk + c * 16);
+      cp_async_16(dst + RAW + c * 16, gv + c * 16);
     }
   };
-  int pg = it.tile_begin + warp;
-  if (pg < it.tile_end) fetch(pg, 0);
-  cp_async_commit();
-  if (pg + kShortWarps < it.tile_end) fetch(pg + kShortWarps, 1);
-  cp_async_commit();
+  const int pg0 = it.tile_begin + warp;
+#pragma unroll
+  for (int st = 0; st < kStagesS - 1; ++st) {
+    if (pg0 + st * kShortWarps < it.tile_end) fetch(pg0 + st * kShortWarps, st);
+    cp_async_commit();
+  }
 
   pdl_wait();
 
-  // query rows (token t, head g of the group) -> row t * G + g, fp16 from the projection workspace
+  // query rows (token t, head hq of the group) -> row t * G + hq, fp16 from the projection workspace
   for (int c = threadIdx.x; c < 32 * (HD / 8); c += kShortThreads) {
     const int row = c / (HD / 8), ch = c % (HD / 8);
     uint4 v = make_uint4(0, 0, 0, 0);
     if (row < R) {
-      const int t = row / G, g = row % G;
-      const uint16_t* src = p.qkv + static_cast<size_t>(it.tok0 + t) * p.n_qkv + (it.kv_head * G + g) * HD + ch * 8;
+      const int t = row / G, hq = row % G;
+      const uint16_t* src = p.qkv + static_cast<size_t>(it.tok0 + t) * p.n_qkv + (it.kv_head * G + hq) * HD + ch * 8;
       v = *reinterpret_cast<const uint4*>(src);
     }
-    *reinterpret_cast<uint4*>(q_s + row * ROWB + swz(row, ch)) = v;
+    *reinterpret_cast<uint4*>(q_s + (row * HD + ch * 8) * 2) = v;
   }
   __syncthreads();
 
-  // A fragments of the query rows stay in registers
+  // A fragments of the query rows, with the permuted dimension index, stay in registers:
+  // k-step ks = 2 blk + j covers dimensions 32 blk + 8 q + 4 j + {0, 1} (a0, a1) and + {2, 3} (a2, a3)
   uint32_t qa[MT][KS][4];
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      const int mat = lane >> 3;
-      const int row = mt * 16 + (mat & 1) * 8 + (lane & 7);
-      ldsm_x4(smem_u32(q_s + row * ROWB + swz(row, 2 * ks + (mat >> 1))), qa[mt][ks]);
+      const int dim = 32 * (ks >> 1) + 8 * q + 4 * (ks & 1);
+      const uint8_t* r0 = q_s + ((mt * 16 + g) * HD + dim) * 2;
+      const uint8_t* r1 = r0 + 8 * HD * 2;
+      qa[mt][ks][0] = *reinterpret_cast<const uint32_t*>(r0);
+      qa[mt][ks][1] = *reinterpret_cast<const uint32_t*>(r1);
+      qa[mt][ks][2] = *reinterpret_cast<const uint32_t*>(r0 + 4);
+      qa[mt][ks][3] = *reinterpret_cast<const uint32_t*>(r1 + 4);
     }
 
   float o[MT][NT][4];
@@ -151,135 +156,154 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
     for (int nt = 0; nt < NT; ++nt) o[mt][nt][0] = o[mt][nt][1] = o[mt][nt][2] = o[mt][nt][3] = 0.f;
   }
 
-  // One page of 16 keys, already widened into k_w / v_w. key_limit: keys at or beyond it are masked; causal: the
-  // page holds the step's own keys key0 .. key0 + 15, and key j is visible to the rows of token t only when j <= t.
-  auto process = [&](int key_limit, bool causal, int key0) {
+  // One page of 16 keys. WIDE = false: kb = K codes (swizzled rows), vb = V^T codes. WIDE = true: the step's own keys
+  // in fp16, kb = K [16][HD], vb = V^T [HD][16], both plain. key_limit: keys at or beyond it are masked; causal: the
+  // page holds the step's keys key0 .. key0 + 15, and key j is visible to the rows of token t only when j <= t.
+  auto process = [&](auto wide_tag, const uint8_t* kb, const uint8_t* vb, int key_limit, bool causal, int key0) {
+    constexpr bool WIDE = decltype(wide_tag)::value;
+    float s[MT][2][2][4];            // [row tile][score tile][k-step parity]
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int par = 0; par < 2; ++par) s[mt][nt][par][0] = s[mt][nt][par][1] = s[mt][nt][par][2] = s[mt][nt][par][3] = 0.f;
+#pragma unroll
+    for (int blk = 0; blk < KS / 2; ++blk)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        const int key = 4 * (g >> 1) + (g & 1) + 2 * nt;
+        uint32_t b[2][2];
+        if (WIDE) {
+          const uint4 w = *reinterpret_cast<const uint4*>(kb + (key * HD + 32 * blk + 8 * q) * 2);
+          b[0][0] = w.x; b[0][1] = w.y; b[1][0] = w.z; b[1][1] = w.w;
+        } else {
+          const int chunk = 2 * blk + (q >> 1);
+          const uint2 w = *reinterpret_cast<const uint2*>(kb + key * HD + ((chunk ^ k_swz<HD>(key)) << 4) + (q & 1) * 8);
+          b[0][0] = e4m3x2_to_f16x2(static_cast<uint16_t>(w.x & 0xffffu));
+          b[0][1] = e4m3x2_to_f16x2(static_cast<uint16_t>(w.x >> 16));
+          b[1][0] = e4m3x2_to_f16x2(static_cast<uint16_t>(w.y & 0xffffu));
+          b[1][1] = e4m3x2_to_f16x2(static_cast<uint16_t>(w.y >> 16));
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          mma_16816(s[mt][nt][0], qa[mt][2 * blk], b[0][0], b[0][1]);
+          mma_16816(s[mt][nt][1], qa[mt][2 * blk + 1], b[1][0], b[1][1]);
+        }
+      }
+    uint32_t pa[MT][4];
+    bool rescale = false;
+    float corr[MT][2];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-      float s[2][4];
-#pragma unroll
-      for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-#pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        uint32_t kb[4];
-        const int mat = lane >> 3;
-        const int key = (mat >> 1) * 8 + (lane & 7);
-        ldsm_x4(smem_u32(k_w + key * ROWB + swz(key, 2 * ks + (mat & 1))), kb);
-        mma_16816(s[0], qa[mt][ks], kb[0], kb[1]);
-        mma_16816(s[1], qa[mt][ks], kb[2], kb[3]);
-      }
-      // mask, running maximum per row (rows lane/4 and lane/4 + 8 of the tile)
-      const int r0 = mt * 16 + (lane >> 2);
+      float sc[2][4];
+      const int r0 = mt * 16 + g;
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const int key = nt * 8 + 2 * (lane & 3) + (e & 1);
+          const int key = 4 * q + (e & 1) + 2 * nt;
           const int row = r0 + (e >> 1) * 8;
           bool vis = key < key_limit;
           if (causal) vis = vis && key0 + key <= row / G;
-          s[nt][e] = vis ? s[nt][e] * p.scale_log2e : kNegBig;
+          sc[nt][e] = vis ? (s[mt][nt][0][e] + s[mt][nt][1][e]) * p.scale_log2e : kNegBig;
         }
-      float mx[2] = {fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1])),
-                     fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]))};
+      float mx[2] = {fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
+                     fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3]))};
+      float sum[2] = {0.f, 0.f};
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
         mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
-      }
-      float corr[2], sum[2] = {0.f, 0.f};
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
         const float m_new = fmaxf(m_run[mt][h], mx[h]);
-        corr[h] = exp2f(m_run[mt][h] - m_new);
+        corr[mt][h] = exp2f(m_run[mt][h] - m_new);
+        rescale = rescale || (m_new != m_run[mt][h]);
         m_run[mt][h] = m_new;
       }
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          // a masked score stays at kNegBig; against a row that has seen nothing yet (m_new == kNegBig) it must
-          // still contribute nothing
-          const float pe = s[nt][e] <= 0.5f * kNegBig ? 0.f : exp2f(s[nt][e] - m_run[mt][e >> 1]);
-          s[nt][e] = pe;
+          // a masked score stays at kNegBig; against a row that has seen nothing yet (reference still kNegBig) it
+          // must contribute nothing all the same
+          const float pe = sc[nt][e] <= 0.5f * kNegBig ? 0.f : exp2f(sc[nt][e] - m_run[mt][e >> 1]);
+          sc[nt][e] = pe;
           sum[e >> 1] += pe;
         }
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         sum[h] += __shfl_xor_sync(0xffffffffu, sum[h], 1);
         sum[h] += __shfl_xor_sync(0xffffffffu, sum[h], 2);
-        l_run[mt][h] = l_run[mt][h] * corr[h] + sum[h];
+        l_run[mt][h] = l_run[mt][h] * corr[mt][h] + sum[h];
       }
-      uint32_t pa[4] = {pack_half2(s[0][0], s[0][1]), pack_half2(s[0][2], s[0][3]), pack_half2(s[1][0], s[1][1]),
-                        pack_half2(s[1][2], s[1][3])};
+      pa[mt][0] = pack_half2(sc[0][0], sc[0][1]);
+      pa[mt][1] = pack_half2(sc[0][2], sc[0][3]);
+      pa[mt][2] = pack_half2(sc[1][0], sc[1][1]);
+      pa[mt][3] = pack_half2(sc[1][2], sc[1][3]);
+    }
+    // the running maxima settle after a few pages: the accumulators are rescaled only when one of them moved
+    if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll
-      for (int nt = 0; nt < NT; nt += 2) {
-        uint32_t vb[4];
-        const int mat = lane >> 3;
-        const int key = (mat & 1) * 8 + (lane & 7);
-        ldsm_x4_trans(smem_u32(v_w + key * ROWB + swz(key, nt + (mat >> 1))), vb);
+      for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          o[mt][nt][e] *= corr[e >> 1];
-          o[mt][nt + 1][e] *= corr[e >> 1];
-        }
-        mma_16816(o[mt][nt], pa, vb[0], vb[1]);
-        mma_16816(o[mt][nt + 1], pa, vb[2], vb[3]);
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) o[mt][nt][e] *= corr[mt][e >> 1];
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      uint32_t b0, b1;
+      if (WIDE) {
+        const uint2 w = *reinterpret_cast<const uint2*>(vb + ((nt * 8 + g) * kPage + 4 * q) * 2);
+        b0 = w.x; b1 = w.y;
+      } else {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(vb + (nt * 8 + g) * kPage + 4 * q);
+        b0 = e4m3x2_to_f16x2(static_cast<uint16_t>(w & 0xffffu));
+        b1 = e4m3x2_to_f16x2(static_cast<uint16_t>(w >> 16));
       }
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) mma_16816(o[mt][nt], pa[mt], b0, b1);
     }
   };
 
   // ------------------------------------------------------------------ cached pages
-  int stage = 0;
-  for (; pg < it.tile_end; pg += kShortWarps) {
-    cp_async_wait<1>();
+  int i = 0;
+  for (int pg = pg0; pg < it.tile_end; pg += kShortWarps, ++i) {
+    cp_async_wait<kStagesS - 2>();
     __syncwarp();
-    // widen the page: a lane takes 16-byte pieces (16 codes) of K and of V and writes two swizzled chunks of halves
-    const uint8_t* rk = raw_of(stage);
-    for (int c = lane; c < 2 * RAW / 16; c += 32) {
-      const bool is_v = c >= RAW / 16;
-      const int cc = is_v ? c - RAW / 16 : c;
-      const uint4 codes = *reinterpret_cast<const uint4*>(rk + (is_v ? RAW : 0) + cc * 16);
-      const int key = cc / (HD / 16), ch = cc % (HD / 16);
-      const uint32_t w[4] = {codes.x, codes.y, codes.z, codes.w};
-      uint32_t h[8];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        h[2 * j] = e4m3x2_to_f16x2(static_cast<uint16_t>(w[j] & 0xffffu));
-        h[2 * j + 1] = e4m3x2_to_f16x2(static_cast<uint16_t>(w[j] >> 16));
-      }
-      uint8_t* dst = (is_v ? v_w : k_w) + key * ROWB;
-      *reinterpret_cast<uint4*>(dst + swz(key, 2 * ch)) = make_uint4(h[0], h[1], h[2], h[3]);
-      *reinterpret_cast<uint4*>(dst + swz(key, 2 * ch + 1)) = make_uint4(h[4], h[5], h[6], h[7]);
-    }
-    __syncwarp();
-    // the raw stage is free again: request the page after next
-    if (pg + 2 * kShortWarps < it.tile_end) fetch(pg + 2 * kShortWarps, stage);
+    // the stage read in the previous round is free: request the page kStagesS - 1 rounds ahead
+    const int ahead = pg + (kStagesS - 1) * kShortWarps;
+    if (ahead < it.tile_end) fetch(ahead, (i + kStagesS - 1) % kStagesS);
     cp_async_commit();
-    process(it.ctx - pg * kPage, false, 0);
-    __syncwarp();
-    stage ^= 1;
+    const uint8_t* st = my + (i % kStagesS) * STAGE;
+    process(std::false_type{}, st, st + RAW, it.ctx - pg * kPage, false, 0);
   }
   cp_async_wait<0>();
 
   // ------------------------------------------------------------------ the step's own keys (last piece, warp 0)
   const bool last_piece = it.slot == it.slot0 + it.n_splits - 1;
   if (last_piece && warp == 0) {
+    uint8_t* k_n = my;                       // [16 keys][HD] fp16
+    uint8_t* v_n = my + kPage * HD * 2;      // [HD][16 keys] fp16
     for (int key0 = 0; key0 < it.n_new; key0 += kPage) {       // up to two pages of them (32 rows, one head per group)
       __syncwarp();
-      for (int c = lane; c < 2 * kPage * (HD / 8); c += 32) {
-        const bool is_v = c >= kPage * (HD / 8);
-        const int cc = is_v ? c - kPage * (HD / 8) : c;
-        const int key = cc / (HD / 8), ch = cc % (HD / 8);
-        uint4 v = make_uint4(0, 0, 0, 0);
+      for (int c = lane; c < kPage * (HD / 8); c += 32) {
+        const int key = c / (HD / 8), ch = c % (HD / 8);
+        uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
         if (key0 + key < it.n_new) {
-          const int col = (p.n_q_heads + (is_v ? p.n_kv_heads : 0) + it.kv_head) * HD + ch * 8;
-          v = *reinterpret_cast<const uint4*>(p.qkv + static_cast<size_t>(it.tok0 + key0 + key) * p.n_qkv + col);
+          const uint16_t* row = p.qkv + static_cast<size_t>(it.tok0 + key0 + key) * p.n_qkv;
+          kv4 = *reinterpret_cast<const uint4*>(row + (p.n_q_heads + it.kv_head) * HD + ch * 8);
+          vv4 = *reinterpret_cast<const uint4*>(row + (p.n_q_heads + p.n_kv_heads + it.kv_head) * HD + ch * 8);
         }
-        *reinterpret_cast<uint4*>((is_v ? v_w : k_w) + key * ROWB + swz(key, ch)) = v;
+        *reinterpret_cast<uint4*>(k_n + (key * HD + ch * 8) * 2) = kv4;
+        const uint32_t vw[4] = {vv4.x, vv4.y, vv4.z, vv4.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          *reinterpret_cast<uint16_t*>(v_n + ((ch * 8 + j) * kPage + key) * 2) =
+              static_cast<uint16_t>(j & 1 ? vw[j >> 1] >> 16 : vw[j >> 1] & 0xffffu);
       }
       __syncwarp();
-      process(it.n_new - key0, true, key0);
+      process(std::true_type{}, k_n, v_n, it.n_new - key0, true, key0);
     }
   }
   __syncthreads();
@@ -289,8 +313,8 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
   float* pml = reinterpret_cast<float*>(q_s);                                    // [warp][32 rows][2], over the queries
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt) {
-    const int r0 = mt * 16 + (lane >> 2);
-    if ((lane & 3) == 0) {
+    const int r0 = mt * 16 + g;
+    if (q == 0) {
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         pml[(warp * 32 + r0 + h * 8) * 2] = m_run[mt][h];
@@ -301,7 +325,7 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
       for (int e = 0; e < 4; ++e)
-        po[(static_cast<size_t>(warp) * 16 * MT + r0 + (e >> 1) * 8) * HD + nt * 8 + 2 * (lane & 3) + (e & 1)] = o[mt][nt][e];
+        po[(static_cast<size_t>(warp) * 16 * MT + r0 + (e >> 1) * 8) * HD + nt * 8 + 2 * q + (e & 1)] = o[mt][nt][e];
   }
   __syncthreads();
   for (int idx = threadIdx.x; idx < R * HD; idx += kShortThreads) {
@@ -317,8 +341,8 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
       L += f * pml[(w * 32 + row) * 2 + 1];
     }
     if (it.n_splits == 1) {
-      const int t = row / G, g = row % G;
-      reinterpret_cast<__half*>(p.out)[static_cast<size_t>(it.tok0 + t) * (p.n_q_heads * HD) + (it.kv_head * G + g) * HD + d] =
+      const int t = row / G, hq = row % G;
+      reinterpret_cast<__half*>(p.out)[static_cast<size_t>(it.tok0 + t) * (p.n_q_heads * HD) + (it.kv_head * G + hq) * HD + d] =
           __float2half_rn(acc / L);
     } else {
       p.part_o[(static_cast<size_t>(it.slot) * 32 + row) * HD + d] = acc;

@@ -141,7 +141,12 @@ __global__ void kv_scatter_u8_kernel(const uint8_t* __restrict__ src_k, const ui
   const size_t dst = ((static_cast<size_t>(page) * n_kv_heads + head) * page_size + slot) * hd + e;
   const size_t src = static_cast<size_t>(t) * n_kv_heads * hd + c * 16;
   *reinterpret_cast<uint4*>(pool_k + dst) = *reinterpret_cast<const uint4*>(src_k + src);
-  *reinterpret_cast<uint4*>(pool_v + dst) = *reinterpret_cast<const uint4*>(src_v + src);
+  // V pages are kept transposed, [hd][page_size]: the short-step attention reads four consecutive keys of one column
+  const uint4 vv = *reinterpret_cast<const uint4*>(src_v + src);
+  const uint32_t w[4] = {vv.x, vv.y, vv.z, vv.w};
+  uint8_t* vt = pool_v + (static_cast<size_t>(page) * n_kv_heads + head) * page_size * hd;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) vt[static_cast<size_t>(e + j) * page_size + slot] = static_cast<uint8_t>(w[j >> 2] >> (8 * (j & 3)));
 }
 
 // In-place re-encoding of bf16 bit patterns as fp16 (same size). Exact for magnitudes in [2^-14, 65504];
