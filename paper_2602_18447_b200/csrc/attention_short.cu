@@ -97,8 +97,7 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
 
   // cached pages of this warp: page_begin + warp, + 4, ...; the copies touch only the cache and the page table, which
   // no kernel of the pass writes, so the first ones go out before the wait on the previous kernel
-  auto fetch = [&](int pg, int stage) {
-    const int32_t id = __ldg(table + pg);
+  auto fetch = [&](int32_t id, int stage) {
     const uint8_t* gk = pool_k + static_cast<size_t>(id) * page_stride + head_off;
     const uint8_t* gv = pool_v + static_cast<size_t>(id) * page_stride + head_off;
     uint8_t* dst = my + stage * STAGE;
@@ -109,11 +108,17 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
     }
   };
   const int pg0 = it.tile_begin + warp;
+  // page ids are read one round before the copies that need them, so that the look-up never stalls the stream
+  int32_t ids[kStagesS];
+#pragma unroll
+  for (int st = 0; st < kStagesS; ++st)
+    ids[st] = pg0 + st * kShortWarps < it.tile_end ? __ldg(table + pg0 + st * kShortWarps) : 0;
 #pragma unroll
   for (int st = 0; st < kStagesS - 1; ++st) {
-    if (pg0 + st * kShortWarps < it.tile_end) fetch(pg0 + st * kShortWarps, st);
+    if (pg0 + st * kShortWarps < it.tile_end) fetch(ids[st], st);
     cp_async_commit();
   }
+  int32_t id_ahead = ids[kStagesS - 1];
 
   pdl_wait();
 
@@ -273,8 +278,9 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
     __syncwarp();
     // the stage read in the previous round is free: request the page kStagesS - 1 rounds ahead
     const int ahead = pg + (kStagesS - 1) * kShortWarps;
-    if (ahead < it.tile_end) fetch(ahead, (i + kStagesS - 1) % kStagesS);
+    if (ahead < it.tile_end) fetch(id_ahead, (i + kStagesS - 1) % kStagesS);
     cp_async_commit();
+    if (ahead + kShortWarps < it.tile_end) id_ahead = __ldg(table + ahead + kShortWarps);
     const uint8_t* st = my + (i % kStagesS) * STAGE;
     process(std::false_type{}, st, st + RAW, it.ctx - pg * kPage, false, 0);
   }
