@@ -41,6 +41,13 @@ __device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint16_t v) {
   asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(v));
   return r;
 }
+// 2^x for x <= 0 by the special-function unit alone; results below the normal range flush to zero, which is what a
+// probability that small contributes anyway.
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
   __half2 h = __floats2half2_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
@@ -166,13 +173,11 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
   // page holds the step's keys key0 .. key0 + 15, and key j is visible to the rows of token t only when j <= t.
   auto process = [&](auto wide_tag, const uint8_t* kb, const uint8_t* vb, int key_limit, bool causal, int key0) {
     constexpr bool WIDE = decltype(wide_tag)::value;
-    float s[MT][2][2][4];            // [row tile][score tile][k-step parity]
+    float s[MT][2][4];               // [row tile][score tile]
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-      for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-        for (int par = 0; par < 2; ++par) s[mt][nt][par][0] = s[mt][nt][par][1] = s[mt][nt][par][2] = s[mt][nt][par][3] = 0.f;
+      for (int nt = 0; nt < 2; ++nt) s[mt][nt][0] = s[mt][nt][1] = s[mt][nt][2] = s[mt][nt][3] = 0.f;
 #pragma unroll
     for (int blk = 0; blk < KS / 2; ++blk)
 #pragma unroll
@@ -192,8 +197,8 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
         }
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          mma_16816(s[mt][nt][0], qa[mt][2 * blk], b[0][0], b[0][1]);
-          mma_16816(s[mt][nt][1], qa[mt][2 * blk + 1], b[1][0], b[1][1]);
+          mma_16816(s[mt][nt], qa[mt][2 * blk], b[0][0], b[0][1]);
+          mma_16816(s[mt][nt], qa[mt][2 * blk + 1], b[1][0], b[1][1]);
         }
       }
     uint32_t pa[MT][4];
@@ -203,15 +208,20 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
     for (int mt = 0; mt < MT; ++mt) {
       float sc[2][4];
       const int r0 = mt * 16 + g;
+      // only the last page of the context and the step's own keys have anything to mask
+      const bool masked = causal || key_limit < kPage;
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const int key = 4 * q + (e & 1) + 2 * nt;
-          const int row = r0 + (e >> 1) * 8;
-          bool vis = key < key_limit;
-          if (causal) vis = vis && key0 + key <= row / G;
-          sc[nt][e] = vis ? (s[mt][nt][0][e] + s[mt][nt][1][e]) * p.scale_log2e : kNegBig;
+          sc[nt][e] = s[mt][nt][e] * p.scale_log2e;
+          if (masked) {
+            const int key = 4 * q + (e & 1) + 2 * nt;
+            const int row = r0 + (e >> 1) * 8;
+            bool vis = key < key_limit;
+            if (causal) vis = vis && key0 + key <= row / G;
+            if (!vis) sc[nt][e] = kNegBig;
+          }
         }
       float mx[2] = {fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
                      fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3]))};
@@ -221,7 +231,7 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
         mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
         mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
         const float m_new = fmaxf(m_run[mt][h], mx[h]);
-        corr[mt][h] = exp2f(m_run[mt][h] - m_new);
+        corr[mt][h] = fast_exp2(m_run[mt][h] - m_new);
         rescale = rescale || (m_new != m_run[mt][h]);
         m_run[mt][h] = m_new;
       }
@@ -229,9 +239,10 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
       for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
+          float pe = fast_exp2(sc[nt][e] - m_run[mt][e >> 1]);
           // a masked score stays at kNegBig; against a row that has seen nothing yet (reference still kNegBig) it
           // must contribute nothing all the same
-          const float pe = sc[nt][e] <= 0.5f * kNegBig ? 0.f : exp2f(sc[nt][e] - m_run[mt][e >> 1]);
+          if (masked && sc[nt][e] <= 0.5f * kNegBig) pe = 0.f;
           sc[nt][e] = pe;
           sum[e >> 1] += pe;
         }
