@@ -70,6 +70,17 @@ def widen_e4m3(codes: np.ndarray) -> np.ndarray:
     return np.where(s == 1, -mag, mag)
 
 
+def widen_e5m2(codes: np.ndarray) -> np.ndarray:
+    """uint8 codes of the 8-bit float with 5 exponent bits (bias 15) and 2 mantissa bits (the other optional 8-bit
+    cache format; it is the upper byte of an fp16) -> float64, exactly: (-1)^s 2^(e-15) (1 + m/4) for 1 <= e <= 30,
+    (-1)^s 2^-14 (m/4) for e = 0; e = 31 is infinity (m = 0) or NaN."""
+    c = np.ascontiguousarray(codes, dtype=np.uint8).astype(np.int64)
+    s, e, m = (c >> 7) & 1, (c >> 2) & 31, c & 3
+    mag = np.where(e == 0, np.ldexp(m / 4.0, -14), np.ldexp(1.0 + m / 4.0, e - 15))
+    mag = np.where(e == 31, np.where(m == 0, np.inf, np.nan), mag)
+    return np.where(s == 1, -mag, mag)
+
+
 # ----------------------------------------------------------------------------------------------
 # model blocks (textbook definitions)
 # ----------------------------------------------------------------------------------------------

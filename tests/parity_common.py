@@ -50,7 +50,7 @@ def oracle_outputs(cfg, weights, batch, steps: Optional[Sequence[int]] = None, t
     else:
         def fn(j, l):
             k, v = context_kv(cfg, idx[j], l, int(batch.ctx_lens[idx[j]]))
-            widen = O.widen_e4m3 if cfg.kv_format == "e4m3" else O.widen_bf16
+            widen = {"e4m3": O.widen_e4m3, "e5m2": O.widen_e5m2}.get(cfg.kv_format, O.widen_bf16)
             return widen(k), widen(v)
     return O.verify_steps(weights, [toks[i] for i in idx], [int(batch.ctx_lens[i]) for i in idx], fn,
                           cfg.verdict_ids, tau)

@@ -267,3 +267,19 @@ def test_e4m3_decode_against_hand_values_and_a_library():
     lib = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
     ours = O.widen_e4m3(np.arange(256, dtype=np.uint8))
     assert np.array_equal(np.isnan(lib), np.isnan(ours)) and np.array_equal(lib[~np.isnan(lib)], ours[~np.isnan(ours)])
+
+
+def test_e5m2_decode_against_hand_values_and_a_library():
+    hand = {0x00: 0.0, 0x01: 2.0 ** -16, 0x03: 3 * 2.0 ** -16, 0x04: 2.0 ** -14, 0x3C: 1.0, 0x3D: 1.25, 0x3E: 1.5,
+            0x40: 2.0, 0x7B: 57344.0, 0xBC: -1.0, 0x38: 0.5}
+    for code, want in hand.items():
+        assert O.widen_e5m2(np.array([code], np.uint8))[0] == want, hex(code)
+    assert np.isinf(O.widen_e5m2(np.array([0x7C], np.uint8))[0]) and np.isnan(O.widen_e5m2(np.array([0x7D], np.uint8))[0])
+    torch = pytest.importorskip("torch")
+    lib = torch.arange(256, dtype=torch.uint8).view(torch.float8_e5m2).to(torch.float64).numpy()
+    ours = O.widen_e5m2(np.arange(256, dtype=np.uint8))
+    assert np.array_equal(np.isnan(lib), np.isnan(ours)) and np.array_equal(lib[~np.isnan(lib)], ours[~np.isnan(ours)])
+    # the upper byte of an fp16
+    h = (np.arange(256, dtype=np.uint16) << 8).view(np.float16).astype(np.float64)
+    ok = ~np.isnan(h)
+    assert np.array_equal(h[ok], ours[ok])

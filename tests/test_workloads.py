@@ -74,3 +74,17 @@ def test_e4m3_encoding_rounds_to_nearest_even_and_saturates():
     assert np.all(same | (zero & ((lib & 0x7F) == 0)))
     # ties go to the even code: 1.0625 is halfway between 1.0 (0x38) and 1.125 (0x39); 1.1875 between 0x39 and 0x3A
     assert e4m3_codes_from_f32(np.array([1.0625, 1.1875, 449.0, 1e9], np.float32)).tolist() == [0x38, 0x3A, 0x7E, 0x7E]
+
+
+def test_e5m2_encoding_rounds_to_nearest_even_and_saturates():
+    from workloads import e5m2_codes_from_f32
+    torch = pytest.importorskip("torch")
+    g = np.random.default_rng(1)
+    x = np.concatenate([g.standard_normal(20000) * 0.78, g.standard_normal(2000) * 1000, [0.0, -0.0, 57344.0, 60000.0,
+                        -1e9, 2.0 ** -17, 3 * 2.0 ** -17, 1.125, 1.375, 2.0 ** -16, 1e-12]]).astype(np.float32)
+    ours = e5m2_codes_from_f32(x)
+    lib = torch.from_numpy(x).clamp(-57344, 57344).to(torch.float8_e5m2).view(torch.uint8).numpy()
+    zero = (ours & 0x7F) == 0
+    assert np.all((ours == lib) | (zero & ((lib & 0x7F) == 0)))
+    # ties to the even code: 1.125 is halfway between 1.0 (0x3C) and 1.25 (0x3D); 1.375 between 0x3D and 0x3E
+    assert e5m2_codes_from_f32(np.array([1.125, 1.375, 60000.0, 1e9], np.float32)).tolist() == [0x3C, 0x3E, 0x7B, 0x7B]

@@ -10,6 +10,7 @@ from .configs import (ModelShape, VerifyConfig, CascadeConfig, CONFIGS, CASCADES
 from .generate import (
     bf16_bits_from_f32,
     e4m3_codes_from_f32,
+    e5m2_codes_from_f32,
     model_weights,
     plant_verdict_rows,
     make_batch,
@@ -21,6 +22,6 @@ from .generate import (
 __all__ = [
     "ModelShape", "VerifyConfig", "CascadeConfig", "CONFIGS", "CASCADES", "get_config", "get_cascade",
     "scaled_config",
-    "bf16_bits_from_f32", "e4m3_codes_from_f32", "model_weights", "plant_verdict_rows", "make_batch",
+    "bf16_bits_from_f32", "e4m3_codes_from_f32", "e5m2_codes_from_f32", "model_weights", "plant_verdict_rows", "make_batch",
     "context_kv", "page_assignment", "Batch",
 ]

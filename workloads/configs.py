@@ -72,7 +72,8 @@ class VerifyConfig:
     # "synthetic": context K/V are drawn i.i.d. N(0, kv_std^2), rounded to bf16, K taken as already rotated.
     ctx_kv: str = "synthetic"
     kv_std: float = 0.78
-    # cache format: "bf16", or "e4m3" (8-bit float, 4 exponent / 3 mantissa bits, unscaled; synthetic contexts only)
+    # cache format: "bf16", or an 8-bit float, unscaled, synthetic contexts only: "e4m3" (4 exponent / 3 mantissa bits)
+    # or "e5m2" (5 / 2: the upper byte of an fp16)
     kv_format: str = "bf16"
     seed: int = 20260218
 
@@ -99,6 +100,9 @@ CONFIGS = {
     "cfg9_q3_short_fp8": VerifyConfig(
         "cfg9_q3_short_fp8", QWEN3_1P7B, 64, ("uniform", 2048, 8192), ("uniform", 1, 4), suffix_len=4, tau=0.9, seed=707,
         kv_format="e4m3"),
+    "cfg10_q3_short_e5m2": VerifyConfig(
+        "cfg10_q3_short_e5m2", QWEN3_1P7B, 64, ("uniform", 2048, 8192), ("uniform", 1, 4), suffix_len=4, tau=0.9,
+        seed=707, kv_format="e5m2"),
     "cfg8_tiny_qknorm": VerifyConfig(
         "cfg8_tiny_qknorm", TINY_QKNORM, 6, ("uniform", 20, 150), ("uniform", 1, 40), tau=0.8, ctx_kv="prefill",
         seed=808),

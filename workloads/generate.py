@@ -58,6 +58,26 @@ def e4m3_codes_from_f32(x: np.ndarray) -> np.ndarray:
     return code.astype(np.uint8) | sign
 
 
+def e5m2_codes_from_f32(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest value of the 8-bit float with 5 exponent bits (bias 15) and 2 mantissa bits (ties to the
+    even code; magnitudes beyond the largest finite value 57344 saturate to it) and return the codes as uint8.
+    Below 2^-14 the format is a fixed-point grid of step 2^-16 (codes 0 .. 4, code 4 being the smallest normal)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32)
+    sign = ((u >> np.uint32(24)) & np.uint32(0x80)).astype(np.uint8)
+    au = u & np.uint32(0x7FFFFFFF)
+    r = au + np.uint32(0xFFFFF)
+    r += (au >> np.uint32(21)) & np.uint32(1)
+    r >>= np.uint32(21)                                   # (fp32 exponent field << 2) | 2 mantissa bits
+    np.minimum(r, np.uint32(((127 - 15) << 2) + 0x7B), out=r)
+    code = r.astype(np.int32) - np.int32((127 - 15) << 2)
+    a = au.view(np.float32)
+    small = a < np.float32(2.0 ** -14)
+    if small.any():
+        code[small] = np.rint(a[small] * np.float32(65536.0)).astype(np.int32)
+    return code.astype(np.uint8) | sign
+
+
 def _normal_bf16(key: Tuple[int, ...], shape: Tuple[int, ...], std: float,
                  pool: Optional[ThreadPoolExecutor] = None) -> np.ndarray:
     """i.i.d. N(0, std^2) rounded to bf16; drawn in fixed row chunks with one stream per chunk."""
@@ -188,17 +208,18 @@ def make_batch(cfg: VerifyConfig, seed: Optional[int] = None) -> Batch:
 
 def context_kv(cfg: VerifyConfig, step: int, layer: int, ctx_len: int,
                seed: Optional[int] = None) -> Tuple[np.ndarray, np.ndarray]:
-    """Synthetic cached K and V of one step for one layer: uint16 bf16 bits (uint8 codes of the 8-bit format when
-    cfg.kv_format == "e4m3": the same draws, rounded once more), each [ctx_len, n_kv_heads, head_dim],
+    """Synthetic cached K and V of one step for one layer: uint16 bf16 bits (uint8 codes of an 8-bit format when
+    cfg.kv_format is "e4m3" or "e5m2": the same draws, rounded once more), each [ctx_len, n_kv_heads, head_dim],
     i.i.d. N(0, kv_std^2). K is taken as already rotated."""
     seed = cfg.seed if seed is None else seed
     m = cfg.model
     shape = (int(ctx_len), m.n_kv_heads, m.head_dim)
     k = _normal_bf16((seed, _TAG_CTXKV, step, layer, 0), shape, cfg.kv_std)
     v = _normal_bf16((seed, _TAG_CTXKV, step, layer, 1), shape, cfg.kv_std)
-    if cfg.kv_format == "e4m3":
+    if cfg.kv_format in ("e4m3", "e5m2"):
         widen = lambda b: (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
-        return e4m3_codes_from_f32(widen(k)), e4m3_codes_from_f32(widen(v))
+        enc = e4m3_codes_from_f32 if cfg.kv_format == "e4m3" else e5m2_codes_from_f32
+        return enc(widen(k)), enc(widen(v))
     return k, v
 
 
