@@ -67,7 +67,7 @@ def work_counts(cfg, batch) -> dict:
     n = batch.step_lens.astype(np.float64)
     c = batch.ctx_lens.astype(np.float64)
     attn_flops_layer = float(np.sum(4.0 * m.n_q_heads * m.head_dim * (n * c + n * (n + 1) / 2)))
-    cell = 1 if getattr(cfg, "kv_format", "bf16") == "e4m3" else 2
+    cell = 1 if getattr(cfg, "kv_format", "bf16") in ("e4m3", "e5m2") else 2
     kv_row = 2 * m.n_kv_heads * m.head_dim * cell                    # bytes of K+V per token per layer
     attn_bytes_layer = float(np.sum(c) * kv_row + T * (m.q_dim + 2 * m.kv_dim + m.q_dim) * 2)
     return {

@@ -115,18 +115,22 @@ int cs_reserve(cs_model* model, int max_steps, int max_tokens);
 int cs_kv_alloc(const cs_model* model, int num_pages, int page_size, int max_seqs, int max_pages_per_seq,
                 void* dev_pool, cs_kv** out);
 /*
- * cs_kv_alloc_e4m3 - the same cache in the optional 8-bit format (no counterpart in the paper, which leaves the
- * cache to its serving engine): one byte per element, the float with 4 exponent bits (bias 7), 3 mantissa bits and
- * no infinities, unscaled; half the bytes, always library-owned (cs_kv_pool_bytes() / 2); pool layout as above
- * except that V pages are kept transposed, [head_dim][page_size].
+ * cs_kv_alloc_8bit - the same cache in an optional 8-bit format (no counterpart in the paper, which leaves the
+ * cache to its serving engine): one byte per element, unscaled, in one of two floating-point formats,
+ *   CS_KV_E4M3  4 exponent bits (bias 7), 3 mantissa bits, no infinities (largest value 448);
+ *   CS_KV_E5M2  5 exponent bits (bias 15), 2 mantissa bits: the upper byte of an fp16.
+ * Half the bytes, always library-owned (cs_kv_pool_bytes() / 2); pool layout as above except that V pages are
+ * kept transposed, [head_dim][page_size].
  * It serves the decode-shaped use of the pass, where reading the cache bounds the time: cs_verify_steps accepts it
  * when every step has at most 32 query rows per kv head (step_lens[i] * n_q_heads / n_kv_heads <= 32; CS_EINVAL
  * otherwise), widens the codes to fp16 on the fly (exact) and computes as with the 16-bit cache. The format is
  * read-only for the pass: contexts come from cs_kv_fill (host arrays of uint8 codes instead of bf16 patterns);
  * cs_prefill and cs_append_accepted return CS_EINVAL on such a cache.
  */
-int cs_kv_alloc_e4m3(const cs_model* model, int num_pages, int page_size, int max_seqs, int max_pages_per_seq,
-                     cs_kv** out);
+#define CS_KV_E4M3 1
+#define CS_KV_E5M2 2
+int cs_kv_alloc_8bit(const cs_model* model, int num_pages, int page_size, int max_seqs, int max_pages_per_seq,
+                     int format, cs_kv** out);
 int cs_kv_free(cs_kv* kv);
 /* Bytes of pool that cs_kv_alloc needs for this geometry (0 on bad arguments). */
 uint64_t cs_kv_pool_bytes(const cs_model* model, int num_pages, int page_size);
@@ -144,7 +148,7 @@ int cs_kv_set_seq(cs_kv* kv, int seq, const int32_t* page_ids, int n_pages, int 
  * cs_kv_fill — write given K/V into the pages of sequence `seq` for one layer (synthetic contexts in
  * tests and benchmarks).
  *   host_k, host_v     host bf16 [ctx_len, n_kv_heads, head_dim] (uint8 codes of the same shape for a cache from
- *                      cs_kv_alloc_e4m3); K already rotated.
+ *                      cs_kv_alloc_8bit); K already rotated.
  * Synchronous on `stream`.
  */
 int cs_kv_fill(cs_kv* kv, int seq, int layer, const uint16_t* host_k, const uint16_t* host_v, void* stream);

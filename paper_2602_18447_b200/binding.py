@@ -15,7 +15,7 @@ CS_OK, CS_EINVAL, CS_ENOMEM, CS_ECUDA, CS_ETIMEOUT, CS_ESTATE, CS_ELIMIT = range
 
 EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_reserve",
-    "cs_kv_alloc", "cs_kv_alloc_e4m3", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
+    "cs_kv_alloc", "cs_kv_alloc_8bit", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
     "cs_verify_steps", "cs_verify_cascade", "cs_append_accepted", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
     "cs_last_status", "cs_selftest_wait_timeout", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
 ]
@@ -67,7 +67,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_model_free": (C.c_int, [vp]),
         "cs_reserve": (C.c_int, [vp, i32, i32]),
         "cs_kv_alloc": (C.c_int, [vp, i32, i32, i32, i32, vp, C.POINTER(vp)]),
-        "cs_kv_alloc_e4m3": (C.c_int, [vp, i32, i32, i32, i32, C.POINTER(vp)]),
+        "cs_kv_alloc_8bit": (C.c_int, [vp, i32, i32, i32, i32, i32, C.POINTER(vp)]),
         "cs_kv_free": (C.c_int, [vp]),
         "cs_kv_pool_bytes": (C.c_uint64, [vp, i32, i32]),
         "cs_kv_set_seq": (C.c_int, [vp, i32, vp, i32, i32]),
@@ -199,10 +199,15 @@ def cs_kv_alloc(model: int, num_pages: int, page_size: int, max_seqs: int, max_p
     return out.value
 
 
-def cs_kv_alloc_e4m3(model: int, num_pages: int, page_size: int, max_seqs: int, max_pages_per_seq: int) -> int:
+CS_KV_E4M3, CS_KV_E5M2 = 1, 2
+
+
+def cs_kv_alloc_8bit(model: int, num_pages: int, page_size: int, max_seqs: int, max_pages_per_seq: int,
+                     fmt: str = "e4m3") -> int:
     out = C.c_void_p()
-    _check(load_library().cs_kv_alloc_e4m3(model, num_pages, page_size, max_seqs, max_pages_per_seq, C.byref(out)),
-           "cs_kv_alloc_e4m3")
+    code = {"e4m3": CS_KV_E4M3, "e5m2": CS_KV_E5M2}[fmt]
+    _check(load_library().cs_kv_alloc_8bit(model, num_pages, page_size, max_seqs, max_pages_per_seq, code,
+                                           C.byref(out)), "cs_kv_alloc_8bit")
     return out.value
 
 
@@ -216,7 +221,7 @@ def cs_kv_set_seq(kv: int, seq: int, page_ids, ctx_len: int) -> None:
 
 
 def cs_kv_fill(kv: int, seq: int, layer: int, host_k: np.ndarray, host_v: np.ndarray, stream=None) -> None:
-    """uint16 arrays (bf16 patterns) for a 16-bit cache, uint8 arrays (codes) for a cache from cs_kv_alloc_e4m3."""
+    """uint16 arrays (bf16 patterns) for a 16-bit cache, uint8 arrays (codes) for a cache from cs_kv_alloc_8bit."""
     dt = np.uint8 if np.asarray(host_k).dtype == np.uint8 else np.uint16
     k = np.ascontiguousarray(host_k, dtype=dt)
     v = np.ascontiguousarray(host_v, dtype=dt)

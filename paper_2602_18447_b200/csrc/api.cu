@@ -113,7 +113,7 @@ struct cs_kv {
   int num_pages, page_size, max_seqs, max_pages_per_seq;
   uint16_t* pool = nullptr;   // 16-bit cells (bf16 values in the fp16 encoding), or 8-bit codes when format == 1
   bool own_pool = false;
-  int format = 0;             // 0: 16-bit cells; 1: 8-bit float, 4 exponent / 3 mantissa bits (read-only for the pass)
+  int format = 0;             // 0: 16-bit cells; CS_KV_E4M3 / CS_KV_E5M2: 8-bit codes (read-only for the pass)
   size_t plane_elems;  // elements of one (layer, K or V) plane
   CUtensorMap tm_pool;
   int32_t* table_host = nullptr;  // pinned [max_seqs, max_pages_per_seq]
@@ -420,11 +420,11 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
     CS_STEP(kProfQkv, gemm_f16_rope(tm_a, lw.tm_wqkv, qkv, T, m->n_qkv, d.d_model, rope_epi, m->status, s));
     ap.k_group_base = (2 * l) * plane_groups;
     ap.v_group_base = (2 * l + 1) * plane_groups;
-    if (kv->format == 1) {
+    if (kv->format != 0) {
       const uint8_t* pool8 = reinterpret_cast<const uint8_t*>(kv->pool);
       CS_STEP(kProfAttn, launch_attention_short(ap, pool8 + static_cast<size_t>(2 * l) * kv->plane_elems,
                                                 pool8 + static_cast<size_t>(2 * l + 1) * kv->plane_elems, d_items,
-                                                L.n_items, L.max_rows, L.any_split, s));
+                                                L.n_items, L.max_rows, L.any_split, kv->format == 2, s));
     } else {
       CS_STEP(kProfAttn, launch_attention(ap, kv->tm_pool, tm_qkv_attn, tm_q3d, d_items, L.n_items, s));
     }
@@ -485,7 +485,7 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
   std::vector<AttnItem> items;
   int n_slots = 0, max_rows = 0;
   bool any_split = false;
-  if (kv->format == 1) {
+  if (kv->format != 0) {
     const int G = m->d.n_q_heads / m->d.n_kv_heads;
     for (int i = 0; i < B; ++i) max_rows = std::max(max_rows, lens[i] * G);
     if (max_rows > 32) return CS_EINVAL;     // the 8-bit cache serves short steps only
@@ -727,9 +727,13 @@ int cs_kv_alloc(const cs_model* m, int num_pages, int page_size, int max_seqs, i
   return kv_alloc_impl(m, num_pages, page_size, max_seqs, max_pages_per_seq, dev_pool, 0, out);
 }
 
-int cs_kv_alloc_e4m3(const cs_model* m, int num_pages, int page_size, int max_seqs, int max_pages_per_seq,
+int cs_kv_alloc_8bit(const cs_model* m, int num_pages, int page_size, int max_seqs, int max_pages_per_seq, int format,
                      cs_kv** out) {
-  return kv_alloc_impl(m, num_pages, page_size, max_seqs, max_pages_per_seq, nullptr, 1, out);
+  if (format != CS_KV_E4M3 && format != CS_KV_E5M2) {
+    if (out) *out = nullptr;
+    return CS_EINVAL;
+  }
+  return kv_alloc_impl(m, num_pages, page_size, max_seqs, max_pages_per_seq, nullptr, format, out);
 }
 
 static int kv_alloc_impl(const cs_model* m, int num_pages, int page_size, int max_seqs, int max_pages_per_seq,
@@ -751,7 +755,7 @@ static int kv_alloc_impl(const cs_model* m, int num_pages, int page_size, int ma
   kv->plane_elems = static_cast<size_t>(num_pages) * m->d.n_kv_heads * page_size * m->d.head_dim;
   kv->ctx_len.assign(max_seqs, -1);
   kv->n_pages.assign(max_seqs, 0);
-  const uint64_t bytes = cs_kv_pool_bytes(m, num_pages, page_size) / (format == 1 ? 2 : 1);
+  const uint64_t bytes = cs_kv_pool_bytes(m, num_pages, page_size) / (format != 0 ? 2 : 1);
   int rc = CS_OK;
   cudaError_t e;
   if (dev_pool) {
@@ -824,7 +828,7 @@ int cs_kv_fill(cs_kv* kv, int seq, int layer, const uint16_t* host_k, const uint
   int rc;
   if ((rc = kv->fill_tmp.ensure(2 * elems * 2))) return rc;
   if ((rc = upload_table(kv, s))) return rc;
-  if (kv->format == 1) {   // 8-bit cache: host_k / host_v hold one code per element
+  if (kv->format != 0) {   // 8-bit cache: host_k / host_v hold one code per element
     uint8_t* tk8 = static_cast<uint8_t*>(kv->fill_tmp.p);
     uint8_t* tv8 = tk8 + elems;
     uint8_t* pool8 = reinterpret_cast<uint8_t*>(kv->pool);

@@ -1,5 +1,5 @@
 // Extend-attention for short steps (at most 32 query rows per kv head: new tokens x heads in the group) over a cache
-// kept in the 8-bit format. With so few rows the pass is bound by reading the cache, not by arithmetic, so the
+// kept in one of the two 8-bit formats. With so few rows the pass is bound by reading the cache, not by arithmetic, so the
 // kernel is organised around bytes: every warp streams whole 16-key pages of one (step, kv head) from global memory
 // with asynchronous copies, three pages in flight, widens the codes to fp16 in registers (exact: every 8-bit value is
 // an fp16 value) and runs the two small products of the page on warp-level tensor-core instructions. There is no wait on
@@ -41,6 +41,20 @@ __device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint16_t v) {
   asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(v));
   return r;
 }
+// Two codes of the 5-exponent-bit format -> two fp16: each code is the upper byte of its fp16. lo = true takes
+// bytes 0, 1 of w, lo = false bytes 2, 3.
+__device__ __forceinline__ uint32_t e5m2x2_to_f16x2(uint32_t w, bool lo) {
+  uint32_t r;
+  if (lo) asm("prmt.b32 %0, %1, %2, 0x1404;" : "=r"(r) : "r"(w), "r"(0u));
+  else    asm("prmt.b32 %0, %1, %2, 0x3424;" : "=r"(r) : "r"(w), "r"(0u));
+  return r;
+}
+// Codes -> fp16 pairs for either 8-bit format (E5M2 = false: 4 exponent / 3 mantissa bits).
+template <bool E5M2>
+__device__ __forceinline__ uint32_t widen2(uint32_t w, bool lo) {
+  if (E5M2) return e5m2x2_to_f16x2(w, lo);
+  return e4m3x2_to_f16x2(static_cast<uint16_t>(lo ? (w & 0xffffu) : (w >> 16)));
+}
 // 2^x for x <= 0 by the special-function unit alone; results below the normal range flush to zero, which is what a
 // probability that small contributes anyway.
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -81,7 +95,7 @@ template <int HD>
 __device__ __forceinline__ int k_swz(int key) { return (((key >> 2) << 1) | (key & 1)) & (HD / 16 - 1); }
 
 // MT = number of 16-row tiles of query rows (1 or 2).
-template <int HD, int MT>
+template <int HD, int MT, bool E5M2>
 __global__ void __launch_bounds__(kShortThreads, MT == 1 ? 3 : 2)
 attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, const uint8_t* __restrict__ pool_v,
                        const AttnItem* __restrict__ items) {
@@ -190,10 +204,10 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
         } else {
           const int chunk = 2 * blk + (q >> 1);
           const uint2 w = *reinterpret_cast<const uint2*>(kb + key * HD + ((chunk ^ k_swz<HD>(key)) << 4) + (q & 1) * 8);
-          b[0][0] = e4m3x2_to_f16x2(static_cast<uint16_t>(w.x & 0xffffu));
-          b[0][1] = e4m3x2_to_f16x2(static_cast<uint16_t>(w.x >> 16));
-          b[1][0] = e4m3x2_to_f16x2(static_cast<uint16_t>(w.y & 0xffffu));
-          b[1][1] = e4m3x2_to_f16x2(static_cast<uint16_t>(w.y >> 16));
+          b[0][0] = widen2<E5M2>(w.x, true);
+          b[0][1] = widen2<E5M2>(w.x, false);
+          b[1][0] = widen2<E5M2>(w.y, true);
+          b[1][1] = widen2<E5M2>(w.y, false);
         }
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
@@ -274,8 +288,8 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
         b0 = w.x; b1 = w.y;
       } else {
         const uint32_t w = *reinterpret_cast<const uint32_t*>(vb + (nt * 8 + g) * kPage + 4 * q);
-        b0 = e4m3x2_to_f16x2(static_cast<uint16_t>(w & 0xffffu));
-        b1 = e4m3x2_to_f16x2(static_cast<uint16_t>(w >> 16));
+        b0 = widen2<E5M2>(w, true);
+        b1 = widen2<E5M2>(w, false);
       }
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) mma_16816(o[mt][nt], pa[mt], b0, b1);
@@ -397,17 +411,17 @@ __global__ void attention_short_merge_kernel(const AttnParams p, const AttnItem*
   }
 }
 
-template <int HD, int MT>
+template <int HD, int MT, bool E5M2>
 cudaError_t launch_short(const AttnParams& p, const uint8_t* pool_k, const uint8_t* pool_v, const AttnItem* items,
                          int n_items, cudaStream_t s) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attention_short_kernel<HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(attention_short_kernel<HD, MT, E5M2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          ShortSmem<HD>::kTotal);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  cudaError_t le = launch_pdl(attention_short_kernel<HD, MT>, dim3(n_items), dim3(kShortThreads), ShortSmem<HD>::kTotal, s,
+  cudaError_t le = launch_pdl(attention_short_kernel<HD, MT, E5M2>, dim3(n_items), dim3(kShortThreads), ShortSmem<HD>::kTotal, s,
                               p, pool_k, pool_v, items);
   count_launch();
   return le != cudaSuccess ? le : cudaGetLastError();
@@ -416,16 +430,17 @@ cudaError_t launch_short(const AttnParams& p, const uint8_t* pool_k, const uint8
 }  // namespace
 
 cudaError_t launch_attention_short(const AttnParams& p, const uint8_t* pool_k, const uint8_t* pool_v,
-                                   const AttnItem* items, int n_items, int max_rows, bool any_split, cudaStream_t s) {
+                                   const AttnItem* items, int n_items, int max_rows, bool any_split, bool e5m2,
+                                   cudaStream_t s) {
   if (n_items <= 0) return cudaSuccess;
   if (max_rows < 1 || max_rows > 32 || (p.head_dim != 64 && p.head_dim != 128)) return cudaErrorInvalidValue;
   cudaError_t e;
-  if (p.head_dim == 128)
-    e = max_rows <= 16 ? launch_short<128, 1>(p, pool_k, pool_v, items, n_items, s)
-                       : launch_short<128, 2>(p, pool_k, pool_v, items, n_items, s);
-  else
-    e = max_rows <= 16 ? launch_short<64, 1>(p, pool_k, pool_v, items, n_items, s)
-                       : launch_short<64, 2>(p, pool_k, pool_v, items, n_items, s);
+#define CS_SHORT(HD_, MT_)                                                               \
+  (e5m2 ? launch_short<HD_, MT_, true>(p, pool_k, pool_v, items, n_items, s)            \
+        : launch_short<HD_, MT_, false>(p, pool_k, pool_v, items, n_items, s))
+  if (p.head_dim == 128) e = max_rows <= 16 ? CS_SHORT(128, 1) : CS_SHORT(128, 2);
+  else e = max_rows <= 16 ? CS_SHORT(64, 1) : CS_SHORT(64, 2);
+#undef CS_SHORT
   if (e != cudaSuccess || !any_split) return e;
   if (p.head_dim == 128)
     e = launch_pdl(attention_short_merge_kernel<128>, dim3(n_items), dim3(128), 0, s, p, items);

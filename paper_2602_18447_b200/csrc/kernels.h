@@ -72,9 +72,10 @@ int attention_max_splits();
 // Short steps over an 8-bit cache (attention_short.cu). Items reuse AttnItem with [tile_begin, tile_end) counted in
 // 16-key PAGES of the cached context; the piece with slot == slot0 + n_splits - 1 also covers the step's own keys.
 // pool_k / pool_v: this layer's planes, K [pages][kv heads][16][head_dim] codes, V [pages][kv heads][head_dim][16]. max_rows = the largest n_new * G of
-// the batch (<= 32). Partial results: part_o [slots][32][head_dim], part_ml [slots][32][2].
+// the batch (<= 32); e5m2 selects the 5-exponent-bit format (else 4 exponent / 3 mantissa bits). Partial results: part_o [slots][32][head_dim], part_ml [slots][32][2].
 cudaError_t launch_attention_short(const AttnParams& p, const uint8_t* pool_k, const uint8_t* pool_v,
-                                   const AttnItem* items, int n_items, int max_rows, bool any_split, cudaStream_t s);
+                                   const AttnItem* items, int n_items, int max_rows, bool any_split, bool e5m2,
+                                   cudaStream_t s);
 // Codes of an 8-bit cache into their pages (V transposed within the page): thread per 16 bytes; rows of src are
 // [n_kv_heads * hd] codes.
 cudaError_t launch_kv_scatter_u8(const uint8_t* src_k, const uint8_t* src_v, int seq, const int32_t* page_table,

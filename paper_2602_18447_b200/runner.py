@@ -38,8 +38,9 @@ class VerifySession:
                     room_for_prefill: bool = False) -> None:
         ps = self.cfg.page_size
         max_pp = max(1, max(len(p) for p in pages_per_step))
-        if getattr(self.cfg, "kv_format", "bf16") == "e4m3":
-            self.kv = B.cs_kv_alloc_e4m3(self.model, total_pages, ps, self.n_steps, max_pp)
+        fmt = getattr(self.cfg, "kv_format", "bf16")
+        if fmt in ("e4m3", "e5m2"):
+            self.kv = B.cs_kv_alloc_8bit(self.model, total_pages, ps, self.n_steps, max_pp, fmt)
         else:
             self.kv = B.cs_kv_alloc(self.model, total_pages, ps, self.n_steps, max_pp)
         for i, pages in enumerate(pages_per_step):

@@ -31,14 +31,15 @@ def _run(cfg, weights, batch, planted=False):
 
 
 def _tiny(name, **kw):
-    base = dict(ctx_kv="synthetic", kv_format="e4m3", suffix_len=0)
+    base = dict(ctx_kv="synthetic", kv_format="e4m3", suffix_len=0)     # kw may choose the other format
     base.update(kw)
     return replace(get_config(name), **base)
 
 
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
 @pytest.mark.parametrize("name,steps", [("cfg1_tiny", ("uniform", 1, 32)), ("cfg8_tiny_qknorm", ("uniform", 1, 16))])
-def test_small_models_every_step(name, steps):
-    cfg = _tiny(name, batch=7, ctx_dist=("uniform", 1, 300), step_dist=steps)
+def test_small_models_every_step(name, steps, fmt):
+    cfg = _tiny(name, batch=7, ctx_dist=("uniform", 1, 300), step_dist=steps, kv_format=fmt)
     stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), planted=True)
     assert stats["logit_err"] < 3e-2
     _run(cfg, model_weights(cfg.model, cfg.seed), make_batch(cfg))
@@ -54,16 +55,18 @@ def test_context_and_step_length_edges(ctx, step):
     _run(cfg, P.planted_weights(cfg), make_batch(cfg), planted=True)
 
 
-def test_long_contexts_cut_into_pieces():
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+def test_long_contexts_cut_into_pieces(fmt):
     """Two steps on contexts of thousands of tokens: every (step, kv head) range is cut into pieces whose partial
     results a second kernel combines."""
-    cfg = _tiny("cfg8_tiny_qknorm", batch=2, ctx_dist=("uniform", 5000, 9000), step_dist=("uniform", 3, 9))
+    cfg = _tiny("cfg8_tiny_qknorm", batch=2, ctx_dist=("uniform", 5000, 9000), step_dist=("uniform", 3, 9), kv_format=fmt)
     stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), planted=True)
     assert stats["logit_err"] < 3e-2
 
 
-def test_decode_shaped_workload_reduced_depth():
-    cfg = scaled_config("cfg9_q3_short_fp8", n_layers=2, batch=9, vocab=20480 + 8)
+@pytest.mark.parametrize("name", ["cfg9_q3_short_fp8", "cfg10_q3_short_e5m2"])
+def test_decode_shaped_workload_reduced_depth(name):
+    cfg = scaled_config(name, n_layers=2, batch=9, vocab=20480 + 8)
     stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), planted=True)
     assert stats["logit_err"] < 3e-2
     _run(cfg, model_weights(cfg.model, cfg.seed), make_batch(cfg))
