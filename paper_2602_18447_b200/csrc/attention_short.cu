@@ -1,7 +1,7 @@
 // Extend-attention for short steps (at most 32 query rows per kv head: new tokens x heads in the group) over a cache
 // kept in one of the two 8-bit formats. With so few rows the pass is bound by reading the cache, not by arithmetic, so the
 // kernel is organised around bytes: every warp streams whole 16-key pages of one (step, kv head) from global memory
-// with asynchronous copies, three pages in flight, widens the codes to fp16 in registers (exact: every 8-bit value is
+// with asynchronous copies, two or three pages in flight, widens the codes to fp16 in registers (exact: every 8-bit value is
 // an fp16 value) and runs the two small products of the page on warp-level tensor-core instructions. There is no wait on
 // another CTA and no spin: pieces of a long context leave partial results that a second kernel combines.
 #include <cuda_fp16.h>
@@ -75,19 +75,22 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
 //    up holding the probabilities of keys 4q .. 4q+3: tile 0 column c is key 4 (c / 2) + c % 2, tile 1 that plus 2.
 //  - V page TRANSPOSED, [HD][16 keys codes] (the layout of the 8-bit pool's V planes): the B operand of
 //    O += P V for output column d and keys 4q .. 4q+3 is one 4-byte load.
-// Shared memory of one warp: kStagesS pages in flight (K codes, 16-byte chunks XOR-swizzled per key row; V^T codes).
-constexpr int kStagesS = 4;
-template <int HD>
+// Shared memory of one warp: kStages pages in flight (K codes, 16-byte chunks XOR-swizzled per key row; V^T codes).
+// One 16-row tile of queries: 3 stages and 4 CTAs per SM; two tiles: 4 stages (the partial results need the room)
+// and 2 CTAs per SM.
+template <int HD, int MT>
 struct ShortSmem {
+  static constexpr int kStages = MT == 1 ? 3 : 4;
   static constexpr int kRawPage = kPage * HD;                  // bytes of one K or V page of one head
   static constexpr int kStage = 2 * kRawPage;
-  static constexpr int kWarp = kStagesS * kStage;
-  static constexpr int kQBytes = 32 * HD * 2;
+  static constexpr int kWarp = kStages * kStage;
+  static constexpr int kQBytes = 16 * MT * HD * 2;
   static constexpr int kTotal = kQBytes + kShortWarps * kWarp;
   // reused after the loop: the step's own keys in fp16 (K [16][HD], V^T [HD][16]) in warp 0's stages, and the
-  // warps' partial results [warp][32 rows][HD] fp32
+  // warps' partial results [warp][16 MT rows][HD] fp32 (+ [warp][32][2] over the queries)
   static_assert(kWarp >= 2 * kPage * HD * 2, "own keys must fit in one warp's stages");
-  static_assert(kShortWarps * kWarp >= kShortWarps * 32 * HD * 4, "partial results must fit");
+  static_assert(kShortWarps * kWarp >= kShortWarps * 16 * MT * HD * 4, "partial results must fit");
+  static_assert(kQBytes >= kShortWarps * 32 * 2 * 4, "row statistics must fit over the queries");
 };
 
 // swizzle of the 16-byte chunks of a K row: distinct for the 8 keys one score tile reads at once
@@ -96,13 +99,14 @@ __device__ __forceinline__ int k_swz(int key) { return (((key >> 2) << 1) | (key
 
 // MT = number of 16-row tiles of query rows (1 or 2).
 template <int HD, int MT, bool E5M2>
-__global__ void __launch_bounds__(kShortThreads, MT == 1 ? 3 : 2)
+__global__ void __launch_bounds__(kShortThreads, MT == 1 ? 4 : 2)
 attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, const uint8_t* __restrict__ pool_v,
                        const AttnItem* __restrict__ items) {
   constexpr int KS = HD / 16;        // k-steps of the score product
   constexpr int NT = HD / 8;         // 8-column tiles of the output
-  constexpr int RAW = ShortSmem<HD>::kRawPage;
-  constexpr int STAGE = ShortSmem<HD>::kStage;
+  constexpr int RAW = ShortSmem<HD, MT>::kRawPage;
+  constexpr int STAGE = ShortSmem<HD, MT>::kStage;
+  constexpr int kStages = ShortSmem<HD, MT>::kStages;
   extern __shared__ __align__(128) uint8_t smem[];
   pdl_launch_dependents();
   const AttnItem it = items[blockIdx.x];
@@ -111,7 +115,7 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
   const int G = p.n_q_heads / p.n_kv_heads;
   const int R = it.n_new * G;                       // query rows in use (<= 16 MT)
   uint8_t* q_s = smem;
-  uint8_t* my = smem + ShortSmem<HD>::kQBytes + warp * ShortSmem<HD>::kWarp;
+  uint8_t* my = smem + ShortSmem<HD, MT>::kQBytes + warp * ShortSmem<HD, MT>::kWarp;
   const int32_t* table = p.page_table + static_cast<size_t>(it.seq) * p.max_pages_per_seq;
   const size_t head_off = static_cast<size_t>(it.kv_head) * kPage * HD;
   const size_t page_stride = static_cast<size_t>(p.n_kv_heads) * kPage * HD;
@@ -130,21 +134,21 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
   };
   const int pg0 = it.tile_begin + warp;
   // page ids are read one round before the copies that need them, so that the look-up never stalls the stream
-  int32_t ids[kStagesS];
+  int32_t ids[kStages];
 #pragma unroll
-  for (int st = 0; st < kStagesS; ++st)
+  for (int st = 0; st < kStages; ++st)
     ids[st] = pg0 + st * kShortWarps < it.tile_end ? __ldg(table + pg0 + st * kShortWarps) : 0;
 #pragma unroll
-  for (int st = 0; st < kStagesS - 1; ++st) {
+  for (int st = 0; st < kStages - 1; ++st) {
     if (pg0 + st * kShortWarps < it.tile_end) fetch(ids[st], st);
     cp_async_commit();
   }
-  int32_t id_ahead = ids[kStagesS - 1];
+  int32_t id_ahead = ids[kStages - 1];
 
   pdl_wait();
 
   // query rows (token t, head hq of the group) -> row t * G + hq, fp16 from the projection workspace
-  for (int c = threadIdx.x; c < 32 * (HD / 8); c += kShortThreads) {
+  for (int c = threadIdx.x; c < 16 * MT * (HD / 8); c += kShortThreads) {
     const int row = c / (HD / 8), ch = c % (HD / 8);
     uint4 v = make_uint4(0, 0, 0, 0);
     if (row < R) {
@@ -299,14 +303,14 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
   // ------------------------------------------------------------------ cached pages
   int i = 0;
   for (int pg = pg0; pg < it.tile_end; pg += kShortWarps, ++i) {
-    cp_async_wait<kStagesS - 2>();
+    cp_async_wait<kStages - 2>();
     __syncwarp();
-    // the stage read in the previous round is free: request the page kStagesS - 1 rounds ahead
-    const int ahead = pg + (kStagesS - 1) * kShortWarps;
-    if (ahead < it.tile_end) fetch(id_ahead, (i + kStagesS - 1) % kStagesS);
+    // the stage read in the previous round is free: request the page kStages - 1 rounds ahead
+    const int ahead = pg + (kStages - 1) * kShortWarps;
+    if (ahead < it.tile_end) fetch(id_ahead, (i + kStages - 1) % kStages);
     cp_async_commit();
     if (ahead + kShortWarps < it.tile_end) id_ahead = __ldg(table + ahead + kShortWarps);
-    const uint8_t* st = my + (i % kStagesS) * STAGE;
+    const uint8_t* st = my + (i % kStages) * STAGE;
     process(std::false_type{}, st, st + RAW, it.ctx - pg * kPage, false, 0);
   }
   cp_async_wait<0>();
@@ -340,7 +344,7 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
   __syncthreads();
 
   // ------------------------------------------------------------------ combine the four warps
-  float* po = reinterpret_cast<float*>(smem + ShortSmem<HD>::kQBytes);           // [warp][16 MT rows][HD]
+  float* po = reinterpret_cast<float*>(smem + ShortSmem<HD, MT>::kQBytes);           // [warp][16 MT rows][HD]
   float* pml = reinterpret_cast<float*>(q_s);                                    // [warp][32 rows][2], over the queries
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt) {
@@ -417,11 +421,11 @@ cudaError_t launch_short(const AttnParams& p, const uint8_t* pool_k, const uint8
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(attention_short_kernel<HD, MT, E5M2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         ShortSmem<HD>::kTotal);
+                                         ShortSmem<HD, MT>::kTotal);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  cudaError_t le = launch_pdl(attention_short_kernel<HD, MT, E5M2>, dim3(n_items), dim3(kShortThreads), ShortSmem<HD>::kTotal, s,
+  cudaError_t le = launch_pdl(attention_short_kernel<HD, MT, E5M2>, dim3(n_items), dim3(kShortThreads), ShortSmem<HD, MT>::kTotal, s,
                               p, pool_k, pool_v, items);
   count_launch();
   return le != cudaSuccess ? le : cudaGetLastError();
