@@ -226,21 +226,25 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
     for (int mt = 0; mt < MT; ++mt) {
       float sc[2][4];
       const int r0 = mt * 16 + g;
-      // only the last page of the context and the step's own keys have anything to mask
-      const bool masked = causal || key_limit < kPage;
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          sc[nt][e] = s[mt][nt][e] * p.scale_log2e;
-          if (masked) {
+        for (int e = 0; e < 4; ++e) sc[nt][e] = s[mt][nt][e] * p.scale_log2e;
+      // Only the last page of the context and the step's own keys have anything to mask (a warp-uniform branch).
+      // A masked score becomes kNegBig and its probability exp2(kNegBig - reference) = 0: the reference is finite,
+      // because every page has a key that all rows see (a context page's first key; the step's first own key).
+      if (causal || key_limit < kPage) {
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
             const int key = 4 * q + (e & 1) + 2 * nt;
             const int row = r0 + (e >> 1) * 8;
             bool vis = key < key_limit;
             if (causal) vis = vis && key0 + key <= row / G;
             if (!vis) sc[nt][e] = kNegBig;
           }
-        }
+      }
       float mx[2] = {fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
                      fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3]))};
       float sum[2] = {0.f, 0.f};
@@ -257,10 +261,7 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
       for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          float pe = fast_exp2(sc[nt][e] - m_run[mt][e >> 1]);
-          // a masked score stays at kNegBig; against a row that has seen nothing yet (reference still kNegBig) it
-          // must contribute nothing all the same
-          if (masked && sc[nt][e] <= 0.5f * kNegBig) pe = 0.f;
+          const float pe = fast_exp2(sc[nt][e] - m_run[mt][e >> 1]);
           sc[nt][e] = pe;
           sum[e >> 1] += pe;
         }
