@@ -265,12 +265,9 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
           sc[nt][e] = pe;
           sum[e >> 1] += pe;
         }
+      // the sums stay per lane (a quarter of each row's keys) until the pages are done
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        sum[h] += __shfl_xor_sync(0xffffffffu, sum[h], 1);
-        sum[h] += __shfl_xor_sync(0xffffffffu, sum[h], 2);
-        l_run[mt][h] = l_run[mt][h] * corr[mt][h] + sum[h];
-      }
+      for (int h = 0; h < 2; ++h) l_run[mt][h] = l_run[mt][h] * corr[mt][h] + sum[h];
       pa[mt][0] = pack_half2(sc[0][0], sc[0][1]);
       pa[mt][1] = pack_half2(sc[0][2], sc[0][3]);
       pa[mt][2] = pack_half2(sc[1][0], sc[1][1]);
@@ -343,6 +340,14 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
     }
   }
   __syncthreads();
+
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      l_run[mt][h] += __shfl_xor_sync(0xffffffffu, l_run[mt][h], 1);
+      l_run[mt][h] += __shfl_xor_sync(0xffffffffu, l_run[mt][h], 2);
+    }
 
   // ------------------------------------------------------------------ combine the four warps
   float* po = reinterpret_cast<float*>(smem + ShortSmem<HD, MT>::kQBytes);           // [warp][16 MT rows][HD]
