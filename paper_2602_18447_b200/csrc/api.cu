@@ -95,10 +95,11 @@ struct cs_model {
   std::vector<void*> owned;
   CUtensorMap tm_lm;
   // workspace
-  DevBuf x, a, qkv, attn_o, hmlp, rope, h_last, lm_part, vlogits, logits, lse, attn_part_o, attn_part_ml, attn_counters;
+  DevBuf x, x_last, a, qkv, attn_o, hmlp, rope, h_last, lm_part, vlogits, logits, lse, attn_part_o, attn_part_ml, attn_counters;
   uint32_t* status = nullptr;
   Staging stg;
   bool keep_logits = false;
+  bool last_rows_compact = false;   // the last run_layers left the steps' final hidden rows in x_last, in step order
   int last_B = 0;
   int64_t last_h2d_bytes = 0;   // bytes the last cs_verify_steps / cs_prefill call copied to the device
   // two-tier pass: list of escalated steps (+ its length) on the draft model, compact results on the target model
@@ -368,6 +369,7 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
                const int32_t* d_tok, cudaStream_t s) {
   const cs_model_desc& d = m->d;
   const int T = L.T;
+  m->last_rows_compact = false;
   const int32_t* d_pos = dev_meta + L.off_pos;
   const int32_t* d_tseq = dev_meta + L.off_tseq;
   const AttnItem* d_items = reinterpret_cast<const AttnItem*>(dev_meta + L.off_items);
@@ -436,6 +438,24 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
                                 d.n_kv_heads, d.head_dim, kPageSize, T, 1, s));
     }
     CS_STEP(kProfO, gemm_f16(tm_o, lw.tm_wo, nullptr, x, T, d.d_model, m->q_dim, kEpiResidAdd, m->status, s));
+    if (l == d.n_layers - 1 && !append_kv) {
+      // Only each step's last position feeds the LM head, and after the last attention no row depends on another:
+      // the last MLP runs on those B rows alone. Same arithmetic per row; the launches are small and bound by
+      // reading the weights, and are timed under "other" so that the per-launch figures of the projection classes
+      // stay those of full launches.
+      float* xl = static_cast<float*>(m->x_last.p);
+      CUtensorMap tm_a_last, tm_h_last;
+      if (!make_gemm_operand_map(&tm_a_last, a, L.B, d.d_model) || !make_gemm_operand_map(&tm_h_last, hmlp, L.B, d.d_ffn)) {
+        g_cuda_error = "cuTensorMapEncodeTiled failed for the last-row buffers";
+        return CS_ECUDA;
+      }
+      CS_STEP(kProfOther, launch_gather_last_rows(x, dev_meta + L.off_cu, xl, L.B, d.d_model, s));
+      CS_STEP(kProfOther, launch_rmsnorm(xl, lw.norm2, a, L.B, d.d_model, d.rms_eps, s));
+      CS_STEP(kProfOther, gemm_f16(tm_a_last, lw.tm_wg, &lw.tm_wu, hmlp, L.B, d.d_ffn, d.d_model, kEpiSwiGLU, m->status, s));
+      CS_STEP(kProfOther, gemm_f16(tm_h_last, lw.tm_wd, nullptr, xl, L.B, d.d_model, d.d_ffn, kEpiResidAdd, m->status, s));
+      m->last_rows_compact = true;
+      break;
+    }
     CS_STEP(kProfNorm, launch_rmsnorm(x, lw.norm2, a, T, d.d_model, d.rms_eps, s));
     CS_STEP(kProfGateUp, gemm_f16(tm_a, lw.tm_wg, &lw.tm_wu, hmlp, T, d.d_ffn, d.d_model, kEpiSwiGLU, m->status, s));
     CS_STEP(kProfDown, gemm_f16(tm_h, lw.tm_wd, nullptr, x, T, d.d_model, d.d_ffn, kEpiResidAdd, m->status, s));
@@ -449,6 +469,7 @@ int ensure_workspace(cs_model* m, int B, int T) {
   const size_t t = static_cast<size_t>(T);
   if ((rc = m->x.ensure(t * d.d_model * 4))) return rc;
   if ((rc = m->a.ensure(t * d.d_model * 2))) return rc;
+  if ((rc = m->x_last.ensure(static_cast<size_t>(B) * d.d_model * 4))) return rc;
   // A 128-row K/V box of the attention kernel may start at any of the T rows: the rows it reaches past the end
   // must exist and be finite (they are masked, but they are multiplied), so the buffer is zeroed when it is made.
   if ((rc = m->qkv.ensure((t + 128) * m->n_qkv * 2, true))) return rc;
@@ -695,7 +716,7 @@ int cs_model_free(cs_model* m) {
   if (!m) return CS_OK;
   cudaDeviceSynchronize();
   for (void* p : m->owned) cudaFree(p);
-  DevBuf* bufs[] = {&m->x, &m->a, &m->qkv, &m->attn_o, &m->hmlp, &m->rope, &m->h_last, &m->lm_part, &m->vlogits,
+  DevBuf* bufs[] = {&m->x, &m->x_last, &m->a, &m->qkv, &m->attn_o, &m->hmlp, &m->rope, &m->h_last, &m->lm_part, &m->vlogits,
                     &m->logits, &m->lse, &m->attn_part_o, &m->attn_part_ml, &m->attn_counters, &m->stg.dev,
                     &m->casc_idx, &m->casc_conf, &m->casc_verdict, &m->casc_accept};
   for (DevBuf* b : bufs) b->release();
@@ -946,7 +967,11 @@ int cs_verify_steps(cs_model* m, const cs_kv* ckv, const int32_t* seq_ids, int B
   float* x = static_cast<float*>(m->x.p);
   uint16_t* h_last = static_cast<uint16_t*>(m->h_last.p);
   const int B_all = ((B + 63) / 64) * 64;
-  CS_STEP(kProfNorm, launch_last_rows_norm(x, dev_meta + L.off_cu, m->final_norm, h_last, B, B_all, d.d_model, d.rms_eps, s));
+  if (m->last_rows_compact)
+    CS_STEP(kProfNorm, launch_last_rows_norm(static_cast<float*>(m->x_last.p), nullptr, m->final_norm, h_last, B, B_all,
+                                             d.d_model, d.rms_eps, s));
+  else
+    CS_STEP(kProfNorm, launch_last_rows_norm(x, dev_meta + L.off_cu, m->final_norm, h_last, B, B_all, d.d_model, d.rms_eps, s));
   CUtensorMap tm_h;
   int tiles_per_cta;
   const int grid = lm_head_grid(d.vocab, &tiles_per_cta);

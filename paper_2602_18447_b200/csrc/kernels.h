@@ -82,7 +82,9 @@ cudaError_t launch_kv_scatter_u8(const uint8_t* src_k, const uint8_t* src_v, int
                                  int max_pages_per_seq, uint8_t* pool_k_plane, uint8_t* pool_v_plane, int n_kv_heads,
                                  int hd, int page_size, int T, cudaStream_t s);
 
-// h[b] = RMSNorm(x[last_row[b]]) as bf16 [B_pad, d]; rows B..B_pad-1 are zeroed.
+// x_last[b] = x[cu_new[b + 1] - 1], fp32 [B, d].
+cudaError_t launch_gather_last_rows(const float* x, const int32_t* cu_new, float* x_last, int B, int d, cudaStream_t s);
+// h[b] = RMSNorm(x[last_row[b]]) as bf16 [B_pad, d]; rows B..B_pad-1 are zeroed. cu_new == nullptr: row b itself.
 cudaError_t launch_last_rows_norm(const float* x, const int32_t* cu_new, const float* gain, uint16_t* h, int B,
                                   int B_pad, int d, float eps, cudaStream_t s);
 // LM head over 128-row vocabulary tiles (tcgen05): per CTA and step the maximum and the sum of exp(z - max)

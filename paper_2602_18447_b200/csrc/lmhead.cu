@@ -222,6 +222,19 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
 }
 
 // One warp per step.
+// x_last[b] = x[last row of step b]: one warp per step.
+__global__ void gather_last_rows_kernel(const float* __restrict__ x, const int32_t* __restrict__ cu_new,
+                                        float* __restrict__ x_last, int B, int d) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B) return;
+  const float4* src = reinterpret_cast<const float4*>(x + static_cast<size_t>(cu_new[b + 1] - 1) * d);
+  float4* dst = reinterpret_cast<float4*>(x_last + static_cast<size_t>(b) * d);
+  for (int i = lane; i < d / 4; i += 32) dst[i] = src[i];
+}
+
 __global__ void last_rows_norm_kernel(const float* __restrict__ x, const int32_t* __restrict__ cu_new,
                                       const float* __restrict__ gain, uint16_t* __restrict__ h, int B, int B_pad,
                                       int d, float eps) {
@@ -235,7 +248,7 @@ __global__ void last_rows_norm_kernel(const float* __restrict__ x, const int32_t
     for (int i = lane; i < d / 4; i += 32) o[i] = make_uint2(0u, 0u);
     return;
   }
-  const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(cu_new[b + 1] - 1) * d);
+  const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(cu_new ? cu_new[b + 1] - 1 : b) * d);
   float ss = 0.f;
   for (int i = lane; i < d / 4; i += 32) {
     const float4 v = xr[i];
@@ -474,6 +487,15 @@ cudaError_t launch_last_rows_norm(const float* x, const int32_t* cu_new, const f
   last_rows_norm_kernel<<<(B_pad + warps - 1) / warps, warps * 32, 0, s>>>(x, cu_new, gain, h, B, B_pad, d, eps);
   count_launch();
   return cudaGetLastError();
+}
+
+cudaError_t launch_gather_last_rows(const float* x, const int32_t* cu_new, float* x_last, int B, int d, cudaStream_t s) {
+  if (B <= 0) return cudaSuccess;
+  const int warps = 4;
+  cudaError_t le = launch_pdl(gather_last_rows_kernel, dim3((B + warps - 1) / warps), dim3(warps * 32), 0, s, x, cu_new,
+                              x_last, B, d);
+  count_launch();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 cudaError_t launch_gate(const float* part_max, const float* part_sum, int n_slices, int nb_stride,
