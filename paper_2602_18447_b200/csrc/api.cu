@@ -422,6 +422,15 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
     CS_STEP(kProfQkv, gemm_f16_rope(tm_a, lw.tm_wqkv, qkv, T, m->n_qkv, d.d_model, rope_epi, m->status, s));
     ap.k_group_base = (2 * l) * plane_groups;
     ap.v_group_base = (2 * l + 1) * plane_groups;
+    if (l == d.n_layers - 1 && append_kv) {
+      // A pass that only appends to the cache has no use for what follows the last layer's K/V projection.
+      CS_STEP(kProfOther, launch_kv_scatter(qkv + m->q_dim, qkv + m->q_dim + m->kv_dim, m->n_qkv, d_tseq, d_pos, 0, 0,
+                                append_kv->table_dev, append_kv->max_pages_per_seq,
+                                append_kv->pool + static_cast<size_t>(2 * l) * append_kv->plane_elems,
+                                append_kv->pool + static_cast<size_t>(2 * l + 1) * append_kv->plane_elems,
+                                d.n_kv_heads, d.head_dim, kPageSize, T, 1, s));
+      break;
+    }
     if (kv->format != 0) {
       const uint8_t* pool8 = reinterpret_cast<const uint8_t*>(kv->pool);
       CS_STEP(kProfAttn, launch_attention_short(ap, pool8 + static_cast<size_t>(2 * l) * kv->plane_elems,
