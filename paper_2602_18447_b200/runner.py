@@ -5,6 +5,7 @@ the smoke check and the benchmark so that all three drive the library the same w
 """
 from __future__ import annotations
 
+import os
 from concurrent.futures import ThreadPoolExecutor
 from typing import List, Optional, Sequence
 
@@ -46,9 +47,10 @@ class VerifySession:
         for i, pages in enumerate(pages_per_step):
             B.cs_kv_set_seq(self.kv, i, pages, 0 if room_for_prefill else int(ctx_lens[i]))
 
-    def fill_synthetic_context(self, context_kv_fn, threads: int = 8) -> None:
+    def fill_synthetic_context(self, context_kv_fn, threads: Optional[int] = None) -> None:
         """context_kv_fn(step, layer) -> (K, V) uint16 arrays [ctx_len, n_kv_heads, head_dim]."""
         jobs = [(i, l) for i in range(self.n_steps) for l in range(self.shape.n_layers)]
+        threads = threads or min(16, os.cpu_count() or 8)
         with ThreadPoolExecutor(max_workers=threads) as pool:
             chunk = 4 * threads
             for o in range(0, len(jobs), chunk):

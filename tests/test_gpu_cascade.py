@@ -199,10 +199,6 @@ def _full_size(target_layers, sample):
         cs.close()
 
 
-def test_1p5b_draft_with_7b_shaped_target_reduced_target_depth():
-    _full_size(target_layers=3, sample=[0, 5, 9, 14])
-
-
 def test_1p5b_draft_with_7b_shaped_target_full_depth():
     """Both models at all 28 layers (3 GB + 15 GB of weights resident together), the whole batch of 16 steps."""
     _full_size(target_layers=None, sample=[5, 14])

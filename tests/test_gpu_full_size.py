@@ -117,17 +117,53 @@ def test_cfg6_second_family_full_depth(weights_q3):
     assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
 
 
-def test_cfg7_short_steps_on_long_contexts_full_depth(weights_q3):
-    """Decode-shaped batch: 64 steps of 5 to 8 new tokens on contexts of 2K to 8K tokens."""
-    cfg, ses, gpu, ref, stats = _run_full("cfg7_q3_short", weights_q3, sample=[0, 33, 63])
-    ses.close()
-    assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
+def test_cfg7_cfg9_short_steps_on_long_contexts_full_depth(weights_q3):
+    """Decode-shaped batch: 64 steps of 5 to 8 new tokens on contexts of 2K to 8K tokens, all 28 layers, over the
+    16-bit cache (cfg7) and over the 8-bit cache holding the same draws rounded to 8 bits (cfg9). The two caches are
+    filled side by side so that the 20 G context values are drawn once."""
+    from concurrent.futures import ThreadPoolExecutor
+    from workloads import context_kv, e4m3_codes_from_f32, page_assignment
+    from paper_2602_18447_b200 import VerifySession, binding as B
+    cfg7, cfg9 = get_config("cfg7_q3_short"), get_config("cfg9_q3_short_fp8")
+    assert cfg7.seed == cfg9.seed and cfg7.model == cfg9.model
+    batch = make_batch(cfg7)
+    sample = [0, 33, 63]
+    sessions = []
+    try:
+        for cfg in (cfg7, cfg9):
+            ses = VerifySession(cfg, weights_q3, batch)
+            sessions.append(ses)
+            B.cs_set_keep_logits(ses.model, True)
+            total, pages = page_assignment(cfg, batch.ctx_lens)
+            ses.alloc_cache(pages, total, batch.ctx_lens)
+        widen = lambda b: (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
 
+        def draw(job):
+            i, l = job
+            k, v = context_kv(cfg7, i, l, int(batch.ctx_lens[i]))
+            return k, v, e4m3_codes_from_f32(widen(k)), e4m3_codes_from_f32(widen(v))
 
-def test_cfg9_short_steps_8bit_cache_full_depth(weights_q3):
-    """The decode-shaped batch over the 8-bit cache (same draws as cfg7, rounded to 8 bits), all 28 layers."""
-    cfg9 = get_config("cfg9_q3_short_fp8")
-    weights = weights_q3 if cfg9.seed == get_config("cfg6_q3_b16").seed else model_weights(cfg9.model, cfg9.seed)
-    cfg, ses, gpu, ref, stats = _run_full("cfg9_q3_short_fp8", weights, sample=[0, 33, 63])
-    ses.close()
-    assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
+        jobs = [(i, l) for i in range(batch.n_steps) for l in range(cfg7.model.n_layers)]
+        import os
+        workers = min(16, os.cpu_count() or 8)
+        with ThreadPoolExecutor(max_workers=workers) as pool:
+            for o in range(0, len(jobs), 4 * workers):
+                part = jobs[o:o + 4 * workers]
+                for (i, l), (k, v, k8, v8) in zip(part, pool.map(draw, part)):
+                    B.cs_kv_fill(sessions[0].kv, i, l, k, v)
+                    B.cs_kv_fill(sessions[1].kv, i, l, k8, v8)
+        # the generator's own 8-bit path gives the same codes as the ones filled above
+        k8, v8 = context_kv(cfg9, 5, 3, int(batch.ctx_lens[5]))
+        k, v = context_kv(cfg7, 5, 3, int(batch.ctx_lens[5]))
+        assert np.array_equal(k8, e4m3_codes_from_f32(widen(k))) and np.array_equal(v8, e4m3_codes_from_f32(widen(v)))
+        for cfg, ses in zip((cfg7, cfg9), sessions):
+            ses.verify()
+            gpu = ses.results()
+            ref = P.oracle_outputs(cfg, weights_q3, batch, steps=sample)
+            stats = P.compare(gpu, ses.last_logits(), ref, cfg.tau, steps=sample, gpu_lse=ses.last_lse())
+            P.check_verdict(gpu, ref, cfg.verdict_ids, steps=sample)
+            assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
+            assert np.all(np.isfinite(gpu["conf"])) and np.all(gpu["conf"] > 0) and np.all(gpu["conf"] <= 1)
+    finally:
+        for ses in sessions:
+            ses.close()
