@@ -156,7 +156,8 @@ int cs_kv_fill(cs_kv* kv, int seq, int layer, const uint16_t* host_k, const uint
 /*
  * cs_prefill — run tokens through the model and APPEND their K/V to the sequences' pages
  * (context management of Algorithm 1, Stage 3: accepted steps become context). The sequences must have
- * enough pages set for ctx_len + lens[i]. On success each sequence's ctx_len grows by lens[i].
+ * enough pages set for ctx_len + lens[i]. On success each sequence's ctx_len grows by lens[i]. The pass ends with
+ * the last layer's K/V projection: nothing reads what would follow it.
  *   seq_ids, lens      host int32[B];  tokens  host int32[sum lens], concatenated per sequence.
  */
 int cs_prefill(cs_model* model, cs_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
@@ -197,6 +198,8 @@ int cs_append_accepted(cs_model* model, cs_kv* kv, int R, const int32_t* req_seq
  *     conf = max_j exp(z[verdict_ids[j]] - logsumexp_v z[v]),   verdict = first j attaining it,
  *     accept = (conf >= tau)     (fp32 comparison; NaN never accepts).
  * The cache is read-only here: K/V of the new tokens live in the model's workspace and are discarded.
+ * Only the last position of a step reaches the LM head, so the MLP half of the last layer is computed for those
+ * B rows alone (same arithmetic per row).
  *   ctx_kv             cache handle whose sequences seq_ids[i] have been set.
  *   seq_ids            host int32[B]. The same sequence may appear several times.
  *   step_tokens        int32[sum step_lens]; host when tokens_on_device == 0 (copied on `stream`), else
