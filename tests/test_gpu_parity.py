@@ -159,3 +159,10 @@ def test_qk_norm_family_reduced_depth(name, layers, batch):
     stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), taus=(0.5,), planted=True)
     assert stats["logit_err"] < 3e-2
     _run(cfg, model_weights(cfg.model, cfg.seed), make_batch(cfg))
+
+
+def test_more_steps_than_one_lm_head_pass_takes():
+    """70 steps: the LM head runs in two passes of at most 64 steps, the last layer's MLP on 70 rows."""
+    cfg = replace(get_config("cfg1_tiny"), batch=70, ctx_dist=("uniform", 0, 90), step_dist=("uniform", 1, 12), suffix_len=2)
+    stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), planted=True)
+    assert stats["logit_err"] < 3e-2 and 0 < ref["accept"].sum() < cfg.batch
