@@ -89,3 +89,13 @@ def test_what_the_format_refuses():
         assert B.cs_take_launch_count() == 0
     finally:
         ses.close()
+
+
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+def test_seven_heads_per_group_two_row_tiles(fmt):
+    """The 7B shape has 7 query heads per kv head: steps of up to 4 tokens fill two 16-row tiles (28 rows) at head
+    dimension 128."""
+    cfg = scaled_config("cfg5_7b_b32", n_layers=1, batch=5, vocab=8192)
+    cfg = replace(cfg, kv_format=fmt, ctx_dist=("uniform", 100, 700), step_dist=("uniform", 1, 2), suffix_len=2)
+    stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), planted=True)
+    assert stats["logit_err"] < 3e-2
