@@ -96,6 +96,17 @@ int cs_model_load(const cs_model_desc* desc, const cs_model_tensors* tensors, in
 int cs_model_free(cs_model* model);
 
 /*
+ * cs_model_set_lm_head_rows - replace rows of a loaded model's LM head, e.g. the rows of the verdict tokens whose
+ * probability is the confidence of Eqs. 2-3 (a verifier whose decision tokens were tuned after the base model was
+ * loaded; the tests use it to give the verdict rows a weight that spreads the confidences over (0, 1)).
+ *   row_ids            host int32[n_rows], each in [0, vocab).
+ *   rows_bf16          host bf16 [n_rows, d_model]; re-encoded like the matrices at load.
+ * Enqueued on `stream` behind earlier passes and synchronised before returning. Errors: CS_EINVAL, CS_ECUDA.
+ */
+int cs_model_set_lm_head_rows(cs_model* model, const int32_t* row_ids, int n_rows, const uint16_t* rows_bf16,
+                              void* stream);
+
+/*
  * cs_reserve — size the per-model activation workspace for batches of up to max_steps steps and
  * max_tokens new tokens in total. Optional: cs_verify_steps / cs_prefill grow the workspace on demand, but
  * growing synchronises the device, so latency-sensitive callers reserve once up front.

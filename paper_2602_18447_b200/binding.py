@@ -14,7 +14,8 @@ from . import build as _build
 CS_OK, CS_EINVAL, CS_ENOMEM, CS_ECUDA, CS_ETIMEOUT, CS_ESTATE, CS_ELIMIT = range(7)
 
 EXPORTED = [
-    "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_reserve",
+    "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_model_set_lm_head_rows",
+    "cs_reserve",
     "cs_kv_alloc", "cs_kv_alloc_8bit", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
     "cs_verify_steps", "cs_verify_cascade", "cs_append_accepted", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
     "cs_last_status", "cs_selftest_wait_timeout", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
@@ -65,6 +66,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_last_cuda_error": (C.c_char_p, []),
         "cs_model_load": (C.c_int, [C.POINTER(cs_model_desc), C.POINTER(cs_model_tensors), i32, C.POINTER(vp)]),
         "cs_model_free": (C.c_int, [vp]),
+        "cs_model_set_lm_head_rows": (C.c_int, [vp, vp, i32, vp, vp]),
         "cs_reserve": (C.c_int, [vp, i32, i32]),
         "cs_kv_alloc": (C.c_int, [vp, i32, i32, i32, i32, vp, C.POINTER(vp)]),
         "cs_kv_alloc_8bit": (C.c_int, [vp, i32, i32, i32, i32, i32, C.POINTER(vp)]),
@@ -181,6 +183,16 @@ def cs_model_load(shape, weights: dict) -> int:
 
 def cs_model_free(model: int) -> None:
     _check(load_library().cs_model_free(model), "cs_model_free")
+
+
+def cs_model_set_lm_head_rows(model: int, row_ids, rows_bf16: np.ndarray, stream=None) -> None:
+    """rows_bf16: uint16 bf16 bit patterns [n_rows, d_model] (host)."""
+    ids = _i32(row_ids)
+    rows = np.ascontiguousarray(rows_bf16, dtype=np.uint16)
+    if rows.ndim != 2 or rows.shape[0] != ids.shape[0]:
+        raise ValueError("rows_bf16 must be [n_rows, d_model]")
+    _check(load_library().cs_model_set_lm_head_rows(model, _np_ptr(ids), int(ids.shape[0]), _np_ptr(rows),
+                                                    _stream_ptr(stream)), "cs_model_set_lm_head_rows")
 
 
 def cs_reserve(model: int, max_steps: int, max_tokens: int) -> None:

@@ -320,6 +320,8 @@ int check_model_desc(const cs_model_desc* d) {
     return CS_EINVAL;
   if (d->head_dim != 64 && d->head_dim != 128) return CS_EINVAL;
   if (d->n_q_heads % d->n_kv_heads) return CS_EINVAL;
+  // a query tile holds the rows of 128 / G tokens for the G query heads of one kv head: G beyond 128 leaves no token
+  if (d->n_q_heads / d->n_kv_heads > 128) return CS_EINVAL;
   if (d->d_model % 8 || d->d_ffn % 8) return CS_EINVAL;
   if (!(d->rope_theta > 0.f) || !(d->rms_eps >= 0.f)) return CS_EINVAL;
   return CS_OK;
@@ -736,6 +738,23 @@ int cs_model_free(cs_model* m) {
     if (m->stg.ev[i]) cudaEventDestroy(m->stg.ev[i]);
   }
   delete m;
+  return CS_OK;
+}
+
+int cs_model_set_lm_head_rows(cs_model* m, const int32_t* row_ids, int n_rows, const uint16_t* rows_bf16, void* stream) {
+  if (!m || n_rows < 0) return CS_EINVAL;
+  if (n_rows == 0) return CS_OK;
+  if (!row_ids || !rows_bf16) return CS_EINVAL;
+  for (int i = 0; i < n_rows; ++i)
+    if (row_ids[i] < 0 || row_ids[i] >= m->d.vocab) return CS_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t dm = static_cast<size_t>(m->d.d_model);
+  for (int i = 0; i < n_rows; ++i) {
+    uint16_t* dst = m->lm_head + static_cast<size_t>(row_ids[i]) * dm;
+    CS_CUDA(cudaMemcpyAsync(dst, rows_bf16 + static_cast<size_t>(i) * dm, dm * 2, cudaMemcpyHostToDevice, s));
+    CS_CUDA(launch_bf16_to_f16(dst, dm, s));   // same re-encoding as at load
+  }
+  CS_CUDA(cudaStreamSynchronize(s));            // the host rows may be released on return
   return CS_OK;
 }
 

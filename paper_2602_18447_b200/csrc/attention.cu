@@ -674,12 +674,8 @@ template <int HD>
 cudaError_t launch_hd(const AttnParams& p, const CUtensorMap& tm_pool, const CUtensorMap& tm_kv_new,
                       const CUtensorMap& tm_q3d, const AttnItem* items, int n_items, cudaStream_t s) {
   using L = AttnSmem<HD>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<uint64_t> smem_opted{0};
+  if (cudaError_t e = opt_in_dynamic_smem(attention_kernel<HD>, L::kTotal, smem_opted); e != cudaSuccess) return e;
   cudaError_t le = launch_pdl(attention_kernel<HD>, dim3(n_items), dim3(kAttnThreads), L::kTotal, s, p, tm_pool, tm_kv_new, tm_q3d,
                               items);
   count_launch();

@@ -424,13 +424,10 @@ __global__ void attention_short_merge_kernel(const AttnParams p, const AttnItem*
 template <int HD, int MT, bool E5M2>
 cudaError_t launch_short(const AttnParams& p, const uint8_t* pool_k, const uint8_t* pool_v, const AttnItem* items,
                          int n_items, cudaStream_t s) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attention_short_kernel<HD, MT, E5M2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         ShortSmem<HD, MT>::kTotal);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<uint64_t> smem_opted{0};
+  if (cudaError_t e = opt_in_dynamic_smem(attention_short_kernel<HD, MT, E5M2>, ShortSmem<HD, MT>::kTotal, smem_opted);
+      e != cudaSuccess)
+    return e;
   cudaError_t le = launch_pdl(attention_short_kernel<HD, MT, E5M2>, dim3(n_items), dim3(kShortThreads), ShortSmem<HD, MT>::kTotal, s,
                               p, pool_k, pool_v, items);
   count_launch();

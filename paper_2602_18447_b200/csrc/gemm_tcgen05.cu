@@ -472,12 +472,8 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
                    int K, uint32_t* status, cudaStream_t stream, const RopeEpilogue& rope = RopeEpilogue{nullptr, 0, 0}) {
   using L = GemmSmem<BN>;
   constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_f16_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<uint64_t> smem_opted{0};
+  if (cudaError_t e = opt_in_dynamic_smem(gemm_f16_kernel<BN, EPI>, L::kTotal, smem_opted); e != cudaSuccess) return e;
   const int m_tiles = (M + BM - 1) / BM;
   const int n_tiles = (N + OUT_BN - 1) / OUT_BN;
   const int kblocks = (K + BK - 1) / BK;

@@ -5,9 +5,26 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 namespace cs {
 
 constexpr int kNumSMs = 148;
+
+// Opt-in to more than 48 KB of dynamic shared memory. cudaFuncSetAttribute applies to the CURRENT device only, so
+// the "already done" flag is kept per device (one bit each; devices beyond 63 simply set the attribute every time).
+// Setting it twice is harmless, so two host threads racing on the first call need no lock.
+template <typename Kernel>
+cudaError_t opt_in_dynamic_smem(Kernel kernel, int bytes, std::atomic<uint64_t>& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && (done.load(std::memory_order_relaxed) >> dev & 1ull)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && tracked) done.fetch_or(1ull << dev, std::memory_order_relaxed);
+  return e;
+}
 
 // One unit of attention work: the query rows of 128 / G consecutive new tokens of one step for the G query
 // heads of one kv head (row = token * G + head-in-group, at most 128 rows), over a range of 128-key tiles.

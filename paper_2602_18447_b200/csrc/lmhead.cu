@@ -433,12 +433,8 @@ __global__ void cascade_select_kernel(const uint8_t* __restrict__ trusted, const
 template <int NB>
 cudaError_t launch_lm_nb(const CUtensorMap& tm_w, const CUtensorMap& tm_h, const LmArgs& a, int grid, cudaStream_t s) {
   using L = LmSmem<NB>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(lm_head_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<uint64_t> smem_opted{0};
+  if (cudaError_t e = opt_in_dynamic_smem(lm_head_kernel<NB>, L::kTotal, smem_opted); e != cudaSuccess) return e;
   cudaError_t le = launch_pdl(lm_head_kernel<NB>, dim3(grid), dim3(kLmThreads), L::kTotal, s, tm_w, tm_h, a);
   count_launch();
   return le != cudaSuccess ? le : cudaGetLastError();

@@ -76,43 +76,78 @@ def compare(gpu: dict, gpu_logits: Optional[np.ndarray], ref: dict, tau: float, 
     assert np.all((acc == 0) | (acc == 1))
     stats["n_near_tau"] = int(near.sum())
     stats["n_accept"] = int(ref["accept"].sum())
+    record_stats("base", stats)
     return stats
 
 
-def compare_planted(gpu: dict, gpu_logits: np.ndarray, ref: dict, tau: float, cfg, weights,
-                    steps: Optional[Sequence[int]] = None) -> dict:
-    """Tolerances for the planted-verdict variant of a workload.
+# Planted-verdict variant: tolerances of the two planted LM-head rows and of the confidence they produce.
+#
+# The planted rows have norm beta ~ ln V + 0.5 instead of init_std * sqrt(d), so the same direction error of the last
+# hidden state (the fp16 rounding of the activations, accumulated over the layers) moves their logits further than an
+# ordinary row's. The bounds below are not derived from that worst case: they are at most three times the largest
+# error observed on the GPU for the class of model (see the table of observed maxima in the design notes), so a
+# regression of the forward pass by a small factor fails them. Keys: (shallow, deep) = (up to 3 layers, more).
+PLANTED_LOGIT_TOL = {"shallow": 4.5e-2, "deep": 2.4e-1}
+PLANTED_CONF_TOL = {"shallow": 5e-3, "deep": 2.5e-2}
 
-    The two planted LM-head rows have norm beta ~ ln V + 0.5 instead of init_std * sqrt(d), so the same
-    direction error of the last hidden state (the fp16 rounding of the activations) moves their logits
-    `row_scale` times further than a random-init row's. The forward is therefore held to 3e-2 on the ordinary
-    rows and to 3e-2 * row_scale on the planted rows, and the softmax / confidence / gate stage is checked
-    tightly on its own: against the oracle's confidence and mask computed from the GPU's own logits."""
+
+def planted_tols(cfg):
+    k = "shallow" if cfg.model.n_layers <= 3 else "deep"
+    return PLANTED_LOGIT_TOL[k], PLANTED_CONF_TOL[k]
+
+
+def record_stats(name: str, stats: dict) -> None:
+    """Append the observed maxima of one comparison to the file named by CS_PARITY_STATS (if set)."""
+    import json
+    import os
+    path = os.environ.get("CS_PARITY_STATS")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps({"case": name, **{k: (float(v) if isinstance(v, (float, np.floating)) else v)
+                                                 for k, v in stats.items()}}) + "\n")
+
+
+def compare_planted(gpu: dict, gpu_logits: np.ndarray, ref: dict, tau: float, cfg, weights=None,
+                    steps: Optional[Sequence[int]] = None, gpu_lse: Optional[np.ndarray] = None,
+                    need_both_sides: bool = False, case: str = "") -> dict:
+    """Planted-verdict variant of a workload against the oracle: ordinary logits and lse at the specified 3e-2, the two
+    planted rows and the confidence at the tightened bounds above, and the accept/escalate mask against the ORACLE's
+    mask for every step whose oracle confidence is further from tau than the confidence bound - trusted steps included.
+    `need_both_sides` additionally demands that at least one trusted and one escalated step were so compared."""
     sel = slice(None) if steps is None else list(steps)
-    m = cfg.model
     vids = list(cfg.verdict_ids)
-    row_norm = np.sqrt((O.widen_bf16(weights["lm_head"][vids[0]]) ** 2).sum())
-    row_scale = max(1.0, row_norm / (m.init_std * np.sqrt(m.d_model)))
+    logit_tol, conf_tol = planted_tols(cfg)
     z = gpu_logits[sel].astype(np.float64)
     d = np.abs(z - ref["logits"])
-    stats = {"planted_logit_err": float(d[:, vids].max()), "logit_err": float(np.delete(d, vids, axis=1).max()),
-             "row_scale": float(row_scale)}
-    assert stats["logit_err"] <= LOGIT_TOL, stats
-    assert stats["planted_logit_err"] <= LOGIT_TOL * row_scale, stats
-    # softmax + confidence + gate, given the logits: tight
-    conf_z, verdict_z, _ = O.verdict_confidence(z, vids)
+    stats = {"planted_logit_err": float(d[:, vids].max()), "logit_err": float(np.delete(d, vids, axis=1).max())}
     conf = gpu["conf"][sel].astype(np.float64)
+    stats["conf_err"] = float(np.max(np.abs(conf - ref["conf"])))
+    if gpu_lse is not None:
+        stats["lse_err"] = float(np.max(np.abs(gpu_lse[sel].astype(np.float64) - ref["lse"])))
+    # softmax + confidence + gate, given the GPU's own logits: tight
+    conf_z, verdict_z, _ = O.verdict_confidence(z, vids)
     stats["conf_err_given_logits"] = float(np.max(np.abs(conf - conf_z)))
-    assert stats["conf_err_given_logits"] <= 1e-4, stats
     acc = gpu["accept"][sel]
+    far = np.abs(ref["conf"] - tau) > conf_tol
+    stats["n_cmp_trusted"] = int((far & (ref["accept"] == 1)).sum())
+    stats["n_cmp_escalated"] = int((far & (ref["accept"] == 0)).sum())
+    stats["n_in_band"] = int((~far).sum())
+    stats["tau"] = float(tau)
+    record_stats(case or cfg.name, stats)
+    assert np.all(np.isfinite(conf)), conf
+    assert stats["logit_err"] <= LOGIT_TOL, stats
+    assert stats["planted_logit_err"] <= logit_tol, stats
+    assert stats["conf_err"] <= conf_tol, stats
+    if gpu_lse is not None:
+        assert stats["lse_err"] <= LOGIT_TOL, stats
+    assert stats["conf_err_given_logits"] <= 1e-4, stats
     sure = np.abs(conf_z - tau) > 1e-4
     assert np.array_equal(acc[sure], O.gate(conf_z, tau)[sure])
-    # against the oracle's own confidence: |d conf| <= |d(z_v - lse)| / 4
-    prop = CONF_TOL + 0.5 * LOGIT_TOL * row_scale
-    stats["conf_err"] = float(np.max(np.abs(conf - ref["conf"])))
-    assert stats["conf_err"] <= prop, stats
-    far = np.abs(ref["conf"] - tau) > prop
-    assert np.array_equal(acc[far], ref["accept"][far])
+    assert np.all((acc == 0) | (acc == 1))
+    # the mask against the oracle's, on both sides of the threshold
+    assert np.array_equal(acc[far], ref["accept"][far]), (acc, ref["accept"], ref["conf"], tau)
+    if need_both_sides:
+        assert stats["n_cmp_trusted"] >= 1 and stats["n_cmp_escalated"] >= 1, stats
     stats["n_accept"] = int(ref["accept"].sum())
     return stats
 
@@ -130,3 +165,36 @@ def planted_weights(cfg, seed=None):
     w = model_weights(cfg.model, cfg.seed if seed is None else seed)
     plant_verdict_rows(w, cfg.verdict_ids, beta=float(np.log(cfg.model.vocab) + 0.5), seed=cfg.seed)
     return w
+
+
+def planted_copy(cfg, weights: dict) -> dict:
+    """The same weights with the planted verdict rows, sharing every tensor but the LM head."""
+    w = dict(weights, lm_head=weights["lm_head"].copy())
+    plant_verdict_rows(w, cfg.verdict_ids, beta=float(np.log(cfg.model.vocab) + 0.5), seed=cfg.seed)
+    return w
+
+
+def sample_both_sides(conf: np.ndarray, tau: float, band: float, n: int, always: Sequence[int] = ()) -> List[int]:
+    """Which steps of a full-size batch the oracle recomputes: picked from the confidences of the pass under test so
+    that the sample has trusted and escalated steps outside the band around tau, the closest ones first (those are
+    the ones a small error would flip), then the extremes. The oracle's own confidences decide the comparison."""
+    conf = np.asarray(conf, dtype=np.float64)
+    above = [int(i) for i in np.argsort(conf) if conf[i] >= tau + band]            # ascending: closest to tau first
+    below = [int(i) for i in np.argsort(-conf) if conf[i] < tau - band]            # descending: closest first
+    picks: List[int] = list(dict.fromkeys(int(i) for i in always))
+    order = []
+    for k in range(max(len(above), len(below))):
+        if k < len(above):
+            order.append(above[k])
+        if k < len(below):
+            order.append(below[k])
+    if above:
+        order.insert(2, above[-1])      # the most confident step
+    if below:
+        order.insert(3, below[-1])      # the least confident step
+    for i in order:
+        if len(picks) >= n:
+            break
+        if i not in picks:
+            picks.append(i)
+    return sorted(picks)

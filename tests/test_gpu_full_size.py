@@ -1,11 +1,13 @@
-"""Parity at the full sizes of the 1.5B-shaped workloads (all 28 layers, the whole batch, the launch configuration
-the benchmark times): the CUDA path runs the complete batch, the CPU oracle recomputes a sample of its steps one by
-one (steps are independent), and the two are compared with the specified tolerances. The tau sweep of the batch-64
-workload goes through cs_escalate_mask on the stored confidences."""
+"""Parity at the full sizes of the workloads (all 28 layers, the whole batch, the launch configuration the benchmark
+times): the CUDA path runs the complete batch, the CPU oracle recomputes a sample of its steps one by one (steps are
+independent), and the two are compared with the specified tolerances. Every workload runs as written (random-init
+weights: every confidence is ~ 1/V and every step escalates) and in its planted-verdict variant, whose confidences
+lie on both sides of the threshold: there the sampled steps include trusted and escalated ones and the mask is held to
+the oracle's. The tau sweep of the batch-64 workload goes through cs_escalate_mask on the planted confidences."""
 import numpy as np
 import pytest
 
-from workloads import get_config, make_batch, model_weights
+from workloads import context_kv, get_config, make_batch, model_weights
 
 import parity_common as P
 
@@ -18,7 +20,19 @@ def weights_1p5b():
     return model_weights(cfg.model, cfg.seed)
 
 
-def _run_full(name, weights, sample):
+def _planted_rows(cfg, weights):
+    """(row ids, bf16 rows) of the planted LM head that differ from the given one."""
+    wp = P.planted_copy(cfg, weights)
+    ids = [int(v) for v in cfg.verdict_ids[:2]]
+    return wp, ids, np.stack([wp["lm_head"][i] for i in ids])
+
+
+def _run_full(name, weights, n_sample, always=()):
+    """The whole batch at full depth, twice in one session: with the weights as specified (random init: every
+    confidence ~ 1/V) and with the two verdict rows of the LM head replaced by the planted ones, which spreads the
+    confidences over (0, 1). The oracle runs its forward once over a sample of steps taken from both sides of the
+    threshold and applies either LM head to it."""
+    from paper_2602_18447_b200 import binding as B
     cfg = get_config(name)
     if weights is None:
         weights = model_weights(cfg.model, cfg.seed)
@@ -28,9 +42,6 @@ def _run_full(name, weights, sample):
         ses.verify()
         gpu = ses.results()
         logits, lse = ses.last_logits(), ses.last_lse()
-        ref = P.oracle_outputs(cfg, weights, batch, steps=sample)
-        stats = P.compare(gpu, logits, ref, cfg.tau, steps=sample, gpu_lse=lse)
-        P.check_verdict(gpu, ref, cfg.verdict_ids, steps=sample)
         # properties that hold for every step of the batch, sampled or not
         assert np.all(np.isfinite(gpu["conf"])) and np.all(gpu["conf"] > 0) and np.all(gpu["conf"] <= 1)
         assert np.array_equal(gpu["accept"], (gpu["conf"] >= np.float32(cfg.tau)).astype(np.uint8))
@@ -39,39 +50,88 @@ def _run_full(name, weights, sample):
         assert np.max(np.abs(lse_from_logits - lse)) < 1e-4          # fused logsumexp == logsumexp of the logits
         vid = list(cfg.verdict_ids)
         assert np.max(np.abs(np.exp(z[:, vid] - lse_from_logits[:, None]).max(axis=1) - gpu["conf"])) < 1e-6
-        return cfg, ses, gpu, ref, stats
+        del z
+
+        # ---- planted verdict rows, same session
+        wp, ids, rows = _planted_rows(cfg, weights)
+        B.cs_model_set_lm_head_rows(ses.model, ids, rows)
+        ses.verify()
+        gpu_p = ses.results()
+        logits_p, lse_p = ses.last_logits(), ses.last_lse()
+        assert np.array_equal(gpu_p["accept"], (gpu_p["conf"] >= np.float32(cfg.tau)).astype(np.uint8))
+        _, conf_tol = P.planted_tols(cfg)
+        sample = P.sample_both_sides(gpu_p["conf"], cfg.tau, conf_tol, n_sample, always=always)
+
+        # ---- the oracle: one forward over the sample, both LM heads
+        toks = P.steps_of(batch)
+
+        def kv_fn(j, l):
+            k, v = context_kv(cfg, sample[j], l, int(batch.ctx_lens[sample[j]]))
+            return P.O.widen_bf16(k), P.O.widen_bf16(v)
+
+        xs, _ = P.O.forward_extend(weights, [toks[i] for i in sample], [int(batch.ctx_lens[i]) for i in sample], kv_fn)
+
+        def head(w):
+            zz = P.O.last_position_logits(w, xs)
+            conf, verdict, l = P.O.verdict_confidence(zz, cfg.verdict_ids)
+            return {"logits": zz, "conf": conf, "verdict": verdict, "lse": l, "accept": P.O.gate(conf, cfg.tau)}
+
+        ref = head(weights)
+        stats = P.compare(gpu, logits, ref, cfg.tau, steps=sample, gpu_lse=lse)
+        P.check_verdict(gpu, ref, cfg.verdict_ids, steps=sample)
+        ref_p = head(wp)
+        stats_p = P.compare_planted(gpu_p, logits_p, ref_p, cfg.tau, cfg, steps=sample, gpu_lse=lse_p,
+                                    need_both_sides=True, case=name + "/full-depth planted")
+        P.check_verdict(gpu_p, ref_p, cfg.verdict_ids, steps=sample)
+        P.record_stats(name + "/full-depth base", stats)
+        return cfg, ses, gpu_p, ref_p, sample, stats, stats_p
     except BaseException:
         ses.close()
         raise
 
 
 def test_cfg2_batch16_full_depth(weights_1p5b):
-    cfg, ses, gpu, ref, stats = _run_full("cfg2_1p5b_b16", weights_1p5b, sample=[0, 7, 15])
+    cfg, ses, gpu_p, ref_p, sample, stats, stats_p = _run_full("cfg2_1p5b_b16", weights_1p5b, 8, always=(0, 15))
     ses.close()
     assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
 
 
 def test_cfg3_batch64_full_depth_and_tau_sweep(weights_1p5b):
+    """The threshold sweep of the batch-64 workload goes through cs_escalate_mask on the stored confidences of the
+    planted variant, so the escalation list changes with tau; the sampled steps are held to the oracle's mask at every
+    tau at which they lie outside the confidence bound."""
     import torch
     from paper_2602_18447_b200 import binding as B
-    cfg, ses, gpu, ref, stats = _run_full("cfg3_1p5b_b64", weights_1p5b, sample=[3, 40])
+    cfg, ses, gpu_p, ref_p, sample, stats, stats_p = _run_full("cfg3_1p5b_b64", weights_1p5b, 8, always=(3, 40))
     try:
         n = cfg.batch
+        _, conf_tol = P.planted_tols(cfg)
+        counts, n_tr, n_es = [], 0, 0
         for tau in cfg.taus:
             acc = torch.zeros(n, dtype=torch.uint8, device="cuda")
             idx = torch.full((n,), -1, dtype=torch.int32, device="cuda")
             cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
             B.cs_escalate_mask(ses.out_conf, tau, acc, idx, cnt)
             torch.cuda.synchronize()
-            want_acc, want_idx, want_cnt = P.O.escalate_list(gpu["conf"], tau)
-            assert int(cnt.item()) == want_cnt and np.array_equal(acc.cpu().numpy(), want_acc)
+            want_acc, want_idx, want_cnt = P.O.escalate_list(gpu_p["conf"], tau)
+            got_acc = acc.cpu().numpy()
+            assert int(cnt.item()) == want_cnt and np.array_equal(got_acc, want_acc)
             assert np.array_equal(idx.cpu().numpy()[:want_cnt], want_idx)
+            counts.append(want_cnt)
+            # against the oracle's own confidences, for the sampled steps outside the bound around this tau
+            far = np.abs(ref_p["conf"] - tau) > conf_tol
+            want = P.O.gate(ref_p["conf"], tau)
+            assert np.array_equal(got_acc[sample][far], want[far])
+            n_tr += int((far & (want == 1)).sum())
+            n_es += int((far & (want == 0)).sum())
+        assert counts == sorted(counts) and counts[0] < counts[-1]     # a higher threshold escalates more steps
+        assert 0 < counts[0] and counts[-1] <= n and n_tr >= 1 and n_es >= 1
     finally:
         ses.close()
 
 
 def test_cfg4_long_context_full_depth(weights_1p5b):
-    cfg, ses, gpu, ref, stats = _run_full("cfg4_1p5b_long", weights_1p5b, sample=[1, 6])
+    cfg, ses, gpu_p, ref_p, sample, stats, stats_p = _run_full("cfg4_1p5b_long", weights_1p5b, 4)
     ses.close()
     assert stats["logit_err"] <= P.LOGIT_TOL
 
@@ -99,7 +159,7 @@ def test_cfg5_7b_shape_full_batch_reduced_depth():
 
 def test_cfg5_7b_shape_full_depth():
     """All 28 layers of the 7B-shaped verifier (15 GB of weights), whole batch; the oracle recomputes two steps."""
-    _, ses, gpu, ref, stats = _run_full("cfg5_7b_b32", None, sample=[5, 28])
+    cfg, ses, gpu_p, ref_p, sample, stats, stats_p = _run_full("cfg5_7b_b32", None, 4)
     ses.close()
     assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
 
@@ -112,7 +172,7 @@ def weights_q3():
 
 def test_cfg6_second_family_full_depth(weights_q3):
     """The 1.7B-shaped model of the second family (query/key normalisation, 8 KV heads), all 28 layers."""
-    cfg, ses, gpu, ref, stats = _run_full("cfg6_q3_b16", weights_q3, sample=[2, 11])
+    cfg, ses, gpu_p, ref_p, sample, stats, stats_p = _run_full("cfg6_q3_b16", weights_q3, 4, always=(2,))
     ses.close()
     assert stats["logit_err"] <= P.LOGIT_TOL and stats["conf_err"] <= P.CONF_TOL
 

@@ -14,15 +14,20 @@ import parity_common as P
 pytestmark = pytest.mark.gpu
 
 
-def _run(cfg, weights, batch, taus=None, planted=False):
+def _run(cfg, weights, batch, taus=None, planted=False, both_sides=False):
+    """One pass at cfg.tau and one per extra threshold, each against the oracle. With `both_sides` the planted runs
+    must, over all thresholds together, have compared at least one trusted and one escalated step with the oracle's
+    mask outside the confidence bound."""
     ses = P.build_session(cfg, weights, batch)
     try:
         ses.verify()
         gpu = ses.results()
         logits, lse = ses.last_logits(), ses.last_lse()
         ref = P.oracle_outputs(cfg, weights, batch)
+        n_tr = n_es = 0
         if planted:
-            stats = P.compare_planted(gpu, logits, ref, cfg.tau, cfg, weights)
+            stats = P.compare_planted(gpu, logits, ref, cfg.tau, cfg, weights, gpu_lse=lse)
+            n_tr, n_es = stats["n_cmp_trusted"], stats["n_cmp_escalated"]
         else:
             stats = P.compare(gpu, logits, ref, cfg.tau, gpu_lse=lse)
             P.check_verdict(gpu, ref, cfg.verdict_ids)
@@ -31,15 +36,17 @@ def _run(cfg, weights, batch, taus=None, planted=False):
             g2 = ses.results()
             r2 = dict(ref, accept=P.O.gate(ref["conf"], tau))
             if planted:
-                # logits of this very call: the atomically accumulated projections differ in the last bits
-                # from call to call, and the planted rows magnify that
-                P.compare_planted(g2, ses.last_logits(), r2, tau, cfg, weights)
+                st = P.compare_planted(g2, ses.last_logits(), r2, tau, cfg, weights, gpu_lse=ses.last_lse())
+                n_tr += st["n_cmp_trusted"]
+                n_es += st["n_cmp_escalated"]
             else:
                 P.compare(g2, None, r2, tau)
+        if both_sides:
+            assert n_tr >= 1 and n_es >= 1, (n_tr, n_es, ref["conf"])
         # host-token entry (tokens copied inside the call) gives the same answer
         ses.verify(host_tokens=True)
         g3 = ses.results()
-        # equal up to the order of the atomic accumulation (a changed last bit can flip an fp16 rounding)
+        # equal up to the order of the accumulation of the residual projections' pieces
         assert np.max(np.abs(g3["conf"] - gpu["conf"])) <= 2.5e-3
         return stats, gpu, ref
     finally:
@@ -56,15 +63,16 @@ def test_cfg1_tiny_with_real_prefill():
 def test_cfg1_tiny_planted_verdict_rows_and_tau_sweep():
     cfg = replace(get_config("cfg1_tiny"), batch=24)
     stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), taus=(0.0, 0.5, 0.7, 0.9, 0.95, 0.99, 1.0001),
-                           planted=True)
+                           planted=True, both_sides=True)
     assert 0 < ref["accept"].sum() < cfg.batch           # the gate is exercised on both sides
     assert ref["conf"].max() > 0.9 and ref["conf"].min() < 0.5
 
 
-@pytest.mark.parametrize("name,layers,batch", [("cfg2_1p5b_b16", 2, 5), ("cfg3_1p5b_b64", 1, 9), ("cfg5_7b_b32", 1, 4)])
+@pytest.mark.parametrize("name,layers,batch", [("cfg2_1p5b_b16", 2, 8), ("cfg3_1p5b_b64", 1, 9), ("cfg5_7b_b32", 1, 8)])
 def test_reduced_depth_large_shapes(name, layers, batch):
     cfg = scaled_config(name, n_layers=layers, batch=batch, vocab=20480 + 8)   # ragged vocabulary tail
-    stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), taus=(0.5, 0.99), planted=True)
+    stats, gpu, ref = _run(cfg, P.planted_weights(cfg), make_batch(cfg), taus=(0.3, 0.5, 0.99), planted=True,
+                           both_sides=True)
     assert stats["logit_err"] < 3e-2
     # the same shapes with the weights as specified (random init): the specified tolerances
     _run(cfg, model_weights(cfg.model, cfg.seed), make_batch(cfg))

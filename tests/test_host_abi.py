@@ -49,6 +49,10 @@ def test_binding_declares_signatures_and_pure_host_calls_work(library_path):
         binding.CS_EINVAL
     out = ctypes.c_void_p()
     assert lib.cs_model_load(None, None, 0, ctypes.byref(out)) == binding.CS_EINVAL and not out.value
+    # more than 128 query heads per kv head leaves no room for a token in a 128-row query tile: refused, not looped on
+    desc = binding.cs_model_desc(1, 256, 256, 1, 64, 688, 4096, 1.0e4, 1e-6)
+    assert lib.cs_model_load(ctypes.byref(desc), None, 0, ctypes.byref(out)) == binding.CS_EINVAL and not out.value
+    assert lib.cs_model_set_lm_head_rows(None, None, 1, None, None) == binding.CS_EINVAL
 
 
 def test_missing_library_fails_loudly(tmp_path):

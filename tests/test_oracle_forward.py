@@ -88,17 +88,17 @@ def test_position_shift_invariance_when_cache_is_rerotated(small_case):
     assert np.max(np.abs(bad["logits"][0] - base["logits"][0])) > 1e-3
 
 
-def test_whole_forward_against_transformers_qwen2(small_case):
-    torch = pytest.importorskip("torch")
-    tr = pytest.importorskip("transformers")
-    w, ctx, new = small_case
-    m = SMALL
+def _library_qwen2(w, m):
+    """The `transformers` Qwen2 architecture in float64 with the given weights loaded: a black box."""
+    import torch
+    import transformers as tr
     cfg = tr.Qwen2Config(vocab_size=m.vocab, hidden_size=m.d_model, intermediate_size=m.d_ffn,
                          num_hidden_layers=m.n_layers, num_attention_heads=m.n_q_heads,
                          num_key_value_heads=m.n_kv_heads, rms_norm_eps=m.rms_eps, rope_theta=m.rope_theta,
                          tie_word_embeddings=False, max_position_embeddings=4096,
                          attn_implementation="eager", use_sliding_window=False)
     assert cfg.rope_parameters["rope_theta"] == m.rope_theta
+    assert getattr(cfg, "head_dim", m.head_dim) == m.head_dim
     model = tr.Qwen2ForCausalLM(cfg).double().eval()
     t = lambda bits: torch.from_numpy(O.widen_bf16(bits))
     sd = {"model.embed_tokens.weight": t(w["embed"]), "lm_head.weight": t(w["lm_head"]),
@@ -115,6 +115,47 @@ def test_whole_forward_against_transformers_qwen2(small_case):
         sd[f"model.layers.{li}.post_attention_layernorm.weight"] = torch.from_numpy(l["norm2"].astype(np.float64))
     missing, unexpected = model.load_state_dict(sd, strict=False)
     assert not unexpected and all("rotary" in k or "inv_freq" in k for k in missing), (missing, unexpected)
+    return model
+
+
+def test_two_layers_of_the_1p5b_shape_against_transformers_qwen2():
+    """The oracle at the widths of the benchmarked model - d_model 1536, 12 query heads on 2 kv heads (6 per group),
+    head_dim 128, d_ffn 8960, rotary base 1e6 - against the library, on two layers and a reduced vocabulary: a head
+    mapping or rotary pairing that only holds for the small pin shape (head_dim 16, 2 heads per group) would show."""
+    torch = pytest.importorskip("torch")
+    pytest.importorskip("transformers")
+    from workloads import bf16_bits_from_f32
+    m = ModelShape("pin-1p5b-2l", 2, 1536, 12, 2, 128, 8960, 2048, 1.0e6)
+    w = model_weights(m, seed=31)
+    g = np.random.default_rng(32)
+    for l in w["layers"]:      # weights large enough that attention and the MLP are far from linear
+        for name in ("wq", "wk", "wv", "wo", "wg", "wu", "wd"):
+            std = 1.5 / np.sqrt(l[name].shape[1])
+            l[name] = bf16_bits_from_f32((std * g.standard_normal(l[name].shape)).astype(np.float32))
+    w["lm_head"] = bf16_bits_from_f32((0.05 * g.standard_normal(w["lm_head"].shape)).astype(np.float32))
+    w["embed"] = bf16_bits_from_f32(g.standard_normal(w["embed"].shape).astype(np.float32))
+    _rand_gains(w, 33)
+    ctx = [g.integers(3, m.vocab, size=c).astype(np.int32) for c in (37, 150)]
+    new = [g.integers(3, m.vocab, size=n).astype(np.int32) for n in (9, 20)]
+    model = _library_qwen2(w, m)
+    kv = O.prefill_context(w, ctx, store_bf16=False)
+    ours = O.verify_steps(w, new, [len(c) for c in ctx], lambda i, l: kv[i][l], (1, 2), 0.5)
+    for i in range(len(ctx)):
+        ids = torch.from_numpy(np.concatenate([ctx[i], new[i]]).astype(np.int64))[None]
+        with torch.no_grad():
+            ref = model(input_ids=ids).logits[0, -1].numpy()
+        assert np.max(np.abs(ref - ours["logits"][i])) < 2e-5      # fp32 rotary tables inside the library
+        p = torch.softmax(torch.from_numpy(ref), -1).numpy()
+        assert abs(max(p[1], p[2]) - ours["conf"][i]) < 1e-6
+    assert np.std(ours["logits"]) > 0.5
+
+
+def test_whole_forward_against_transformers_qwen2(small_case):
+    torch = pytest.importorskip("torch")
+    pytest.importorskip("transformers")
+    w, ctx, new = small_case
+    m = SMALL
+    model = _library_qwen2(w, m)
 
     kv = O.prefill_context(w, ctx, store_bf16=False)
     ours = O.verify_steps(w, new, [len(c) for c in ctx], lambda i, l: kv[i][l], (1, 2), 0.5)

@@ -88,3 +88,15 @@ def test_e5m2_encoding_rounds_to_nearest_even_and_saturates():
     assert np.all((ours == lib) | (zero & ((lib & 0x7F) == 0)))
     # ties to the even code: 1.125 is halfway between 1.0 (0x3C) and 1.25 (0x3D); 1.375 between 0x3D and 0x3E
     assert e5m2_codes_from_f32(np.array([1.125, 1.375, 60000.0, 1e9], np.float32)).tolist() == [0x3C, 0x3E, 0x7B, 0x7B]
+
+
+def test_sample_of_a_full_size_batch_has_both_sides_of_the_threshold():
+    """Host logic of the full-size parity tests: which steps the oracle recomputes."""
+    import parity_common as P
+    conf = np.array([0.05, 0.93, 0.999, 0.87, 0.5, 0.91, 0.2, 0.97, 0.895, 0.0001])
+    s = P.sample_both_sides(conf, 0.9, 0.02, 6, always=(4,))
+    assert len(s) == 6 and s == sorted(s) and 4 in s
+    assert 1 in s and 3 in s            # the trusted and the escalated step closest to the band come first
+    assert 2 in s and 9 in s            # then the extremes
+    assert 8 not in s and 5 not in s    # inside the band around tau: never picked
+    assert P.sample_both_sides(np.full(4, 1e-5), 0.9, 0.02, 3) == [0, 1, 2]    # one-sided batches still give a sample
