@@ -5,8 +5,9 @@
     python bench.py --cascade cascade_1p5b_7b [--steps K] [--warmup W]     (two-tier pass, one GPU; see run_cascade)
 
 One "step" is one cs_verify_steps call over the whole batch of the workload (every kernel of the pass).
-Prints ONE JSON line. With --gpus N > 1 (launched by torch.distributed.run) every rank runs an independent
-replica on its own seeded batch: the pass has no exchange step, so there is no collective on the data path.
+Prints ONE JSON line. With --gpus N > 1 every rank runs an independent replica on its own seeded batch (launched by
+torch.distributed.run, or by this script itself when it is started without a launcher): the pass has no exchange
+step, so there is no collective on the data path.
 `--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same workload instead.
 """
 from __future__ import annotations
@@ -33,21 +34,24 @@ DEFAULT_WORKLOAD = "cfg2_1p5b_b16"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
-# DRAM bytes (read + write) of one gate/up GEMM launch of the default workload, from the ncu capture summarised in
-# profiles/gemm_f16_cfg2_4layers.md, and the hash of the kernel source that capture was taken with. A changed kernel
-# has no counters: traffic is then reported as null.
-GATEUP_TRAFFIC = {"workload": "cfg2_1p5b_b16", "bytes": 58.654720e6 + 4.816128e6,
-                  "source": "paper_2602_18447_b200/csrc/gemm_tcgen05.cu", "sha256_16": "14d933d57643dc3b"}
+# DRAM counters of the dominant kernel (one gate/up GEMM launch of the default workload): read from the small JSON that
+# sits beside the ncu summary they were taken for. It names the kernel source and its hash at capture time; a kernel
+# that has changed since has no counters, and traffic is then reported as null.
+COUNTERS_JSON = os.path.join(ROOT, "profiles", "gemm_gateup_cfg2_counters.json")
 
 
 def gateup_traffic(workload: str):
     import hashlib
     try:
-        with open(os.path.join(ROOT, GATEUP_TRAFFIC["source"]), "rb") as f:
+        with open(COUNTERS_JSON) as f:
+            c = json.load(f)
+        with open(os.path.join(ROOT, c["source"]), "rb") as f:
             h = hashlib.sha256(f.read()).hexdigest()[:16]
-    except OSError:
+    except (OSError, KeyError, ValueError):
         return None
-    return GATEUP_TRAFFIC["bytes"] if (workload == GATEUP_TRAFFIC["workload"] and h == GATEUP_TRAFFIC["sha256_16"]) else None
+    if workload != c.get("workload") or h != c.get("sha256_16"):
+        return None
+    return float(c["dram_bytes_read"]) + float(c["dram_bytes_write"])
 
 
 def load_peaks():
@@ -99,7 +103,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", self.uuid], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
@@ -230,6 +234,8 @@ def run_ours(args, cfg):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the pass has no CPU path")
+    if world != args.gpus:
+        raise RuntimeError(f"--gpus {args.gpus} but the launcher started {world} process(es)")
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -260,20 +266,34 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
 
     # ---- device-resident throughput -------------------------------------------------------------
+    # The K-step timed loop is repeated so that the whole timed region lasts seconds: the median repeat is the
+    # reported number (the best one is given beside it) and the clock sampler sees the GPU under the power state that
+    # the loop settles into, not the first milliseconds after idle.
+    def timed_loop():
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for _ in range(K):
+            ses.verify()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+        return ev0.elapsed_time(ev1)
+
     B.cs_take_launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    torch.cuda.synchronize()
+    first = timed_loop()
+    launches = B.cs_take_launch_count()            # of one K-step loop
+    repeats = max(10, min(400, int(np.ceil(args.min_seconds * 1e3 / max(first, 1e-3)))))
+    if world > 1:                                  # every rank must run the same number of loops
+        r = torch.tensor([repeats], dtype=torch.int64, device="cuda")
+        dist.all_reduce(r, op=dist.ReduceOp.MAX)
+        repeats = int(r.item())
     t_wall0 = time.time()
-    ev0.record(stream)
-    for _ in range(K):
-        ses.verify()
-    ev1.record(stream)
-    torch.cuda.synchronize()
+    loop_ms = [timed_loop() for _ in range(repeats)]
     t_wall1 = time.time()
-    barrier()
-    launches = B.cs_take_launch_count()
-    ms = ev0.elapsed_time(ev1)
+    ms = float(np.median(loop_ms))
+    ms_best = float(np.min(loop_ms))
     B.cs_last_status(ses.model)
 
     # ---- end to end: host tokens in, results read back on the host, every step ---------------------
@@ -283,34 +303,50 @@ def run_ours(args, cfg):
         ses.verify(host_tokens=True)
     torch.cuda.synchronize()
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(K):
-        ses.verify(host_tokens=True)
-        conf_host.copy_(ses.out_conf, non_blocking=True)
-        acc_host.copy_(ses.out_accept, non_blocking=True)
-        stream.synchronize()                      # the caller reads the mask before its next step
-    e1.record(stream)
-    torch.cuda.synchronize()
-    barrier()
-    ms_e2e = e0.elapsed_time(e1)
+    e2e_ms = []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(K):
+            ses.verify(host_tokens=True)
+            conf_host.copy_(ses.out_conf, non_blocking=True)
+            acc_host.copy_(ses.out_accept, non_blocking=True)
+            stream.synchronize()                      # the caller reads the mask before its next step
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+        e2e_ms.append(e0.elapsed_time(e1))
+    ms_e2e = float(np.median(e2e_ms))
     h2d_bytes = B.cs_last_h2d_bytes(ses.model)     # tokens + batch metadata, one pinned block per call
 
     # ---- per-kernel durations (events around every launch; same workload, same process) -------------
+    # Read back after every K-step loop (the event pool is reused); repeated like the timed loop, with the clocks
+    # sampled over this region on their own, since these are the times the per-kernel roofline figures come from.
     B.cs_profile(ses.model, True)
-    for _ in range(K):
-        ses.verify()
-    torch.cuda.synchronize()
-    prof = B.cs_profile_read(ses.model)
+    prof = None
+    t_prof0 = time.time()
+    for _ in range(max(3, repeats // 3)):
+        for _ in range(K):
+            ses.verify()
+        torch.cuda.synchronize()
+        part = B.cs_profile_read(ses.model)
+        prof = part if prof is None else {k: (prof[k][0] + v[0], prof[k][1] + v[1]) for k, v in part.items()}
+    t_prof1 = time.time()
     B.cs_profile(ses.model, False)
     sampler.stop()
     clocks = sampler.summary(t_wall0, t_wall1)
+    clocks_prof = sampler.summary(t_prof0, t_prof1)
 
     ms, ms_e2e, all_steps, all_tokens = aggregate_over_ranks(
         ms, ms_e2e, batch.n_steps, batch.n_tokens, device="cuda" if world > 1 else None)
 
+    # Peaks: fp16 and bf16 share the tensor peak. Two measured figures exist: the burst one (cuBLAS timed alone, near
+    # the full clock) and the sustained one (seconds of back-to-back GEMMs under the power cap, ~1.3 GHz). Fractions
+    # are given against the burst figure - the stricter one - with the sustained reading beside it, and each time also
+    # as time x median SM clock so that runs at different clocks can be compared.
     peaks, peak_kind = load_peaks()
-    tensor_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))   # fp16 and bf16 share the peak
+    tensor_peak = float(peaks["bf16_tflops"])
+    tensor_peak_sus = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
     hbm_peak = float(peaks["hbm_gbs"])
 
     def per_launch_ms(name):
@@ -325,10 +361,12 @@ def run_ours(args, cfg):
                         ("gemm_gateup", counts["gemm_gateup_flops"]), ("gemm_down", counts["gemm_down_flops"])):
         t_ms = per_launch_ms(name)
         kernels[name] = {"ms_per_launch": t_ms, "tflops": flops / (t_ms * 1e-3) / 1e12,
-                         "frac_tensor": flops / (t_ms * 1e-3) / 1e12 / tensor_peak}
+                         "frac_tensor": flops / (t_ms * 1e-3) / 1e12 / tensor_peak,
+                         "frac_tensor_sustained": flops / (t_ms * 1e-3) / 1e12 / tensor_peak_sus}
     a_ms = per_launch_ms("attention")
     kernels["attention"] = {"ms_per_launch": a_ms, "tflops": counts["attention_flops"] / (a_ms * 1e-3) / 1e12,
                             "frac_tensor": counts["attention_flops"] / (a_ms * 1e-3) / 1e12 / tensor_peak,
+                            "frac_tensor_sustained": counts["attention_flops"] / (a_ms * 1e-3) / 1e12 / tensor_peak_sus,
                             "gbs": counts["attention_bytes"] / (a_ms * 1e-3) / 1e9,
                             "frac_hbm": counts["attention_bytes"] / (a_ms * 1e-3) / 1e9 / hbm_peak}
     l_ms = per_launch_ms("lm_head")
@@ -336,12 +374,36 @@ def run_ours(args, cfg):
                           "frac_hbm": counts["lm_head_bytes"] / (l_ms * 1e-3) / 1e9 / hbm_peak}
     prof_total = sum(v[0] for v in prof.values())
     shares = {k: (v[0] / prof_total if prof_total else 0.0) for k, v in prof.items()}
+    all_gemm_flops = sum(counts[k] for k in ("gemm_qkv_flops", "gemm_o_flops", "gemm_gateup_flops", "gemm_down_flops"))
+    all_gemm_ms = sum(kernels[k]["ms_per_launch"] for k in ("gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down"))
+    kernels["gemm_all_four"] = {"ms_per_layer": all_gemm_ms, "tflops": all_gemm_flops / (all_gemm_ms * 1e-3) / 1e12,
+                                "frac_tensor": all_gemm_flops / (all_gemm_ms * 1e-3) / 1e12 / tensor_peak,
+                                "frac_tensor_sustained": all_gemm_flops / (all_gemm_ms * 1e-3) / 1e12 / tensor_peak_sus}
+
+    # Whole step against its own roofline: every kernel at the bound that binds it (projections: tensor peak;
+    # attention: the slower of its flops at tensor peak and its bytes at copy bandwidth; LM head: its bytes).
+    def step_roofline_ms(tp):
+        per_layer = all_gemm_flops / (tp * 1e12) + max(counts["attention_flops"] / (tp * 1e12),
+                                                       counts["attention_bytes"] / (hbm_peak * 1e9))
+        return 1e3 * (L * per_layer + counts["lm_head_bytes"] / (hbm_peak * 1e9))
+
+    step_ms = ms / K
+    whole = {"algorithmic_ms": step_roofline_ms(tensor_peak), "algorithmic_ms_sustained": step_roofline_ms(tensor_peak_sus),
+             "measured_ms": step_ms}
+    whole["frac"] = whole["algorithmic_ms"] / step_ms
+    whole["frac_sustained"] = whole["algorithmic_ms_sustained"] / step_ms
+    mhz = clocks.get("sm_mhz")
+    mhz_prof = clocks_prof.get("sm_mhz")
 
     out = {
         "metric": METRIC, "value": all_steps * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16", "data": "synthetic",
         "tokens_per_s": all_tokens * K / (ms * 1e-3),
+        "timing": {"repeats": repeats, "steps_per_repeat": K, "reported": "median repeat", "ms_per_step_median": ms / K,
+                   "ms_per_step_best": ms_best / K, "ms_per_step_worst": float(np.max(loop_ms)) / K,
+                   "ms_x_sm_mhz": (ms / K * mhz) if mhz else None},
+        "whole_step": whole,
         "config": {"workload": cfg.name, "model": cfg.model.name, "layers": cfg.model.n_layers, "batch": cfg.batch, "new_tokens": counts["T"],
                    "ctx_tokens": int(batch.ctx_lens.sum()), "tau": cfg.tau, "page_size": cfg.page_size,
                    "l2": "inputs larger than L2 (3.1 GB of weights streamed every step)",
@@ -349,13 +411,16 @@ def run_ours(args, cfg):
                                  "launches are timed under 'other', not in the per-launch projection figures",
                    "replicas": world},
         "clocks": clocks,
+        "clocks_per_kernel_run": clocks_prof,
         "e2e": {"value": all_steps * K / (ms_e2e * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": int(h2d_bytes),
                 "d2h_bytes_per_step": int(batch.n_steps * 5), "ms_per_step": ms_e2e / K},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "gemm_f16_kernel<256, SwiGLU> (gate/up projection)", "bound": "tensor",
                      "achieved": gu_tf, "peak": tensor_peak, "unit": "TFLOP/s", "frac": gu_tf / tensor_peak,
-                     "peak_kind": f"{peak_kind} bf16 sustained (fp16 has the same nominal peak)",
+                     "peak_kind": f"{peak_kind} bf16 burst (fp16 has the same nominal peak)",
+                     "peak_sustained": tensor_peak_sus, "frac_sustained": gu_tf / tensor_peak_sus,
+                     "ms_x_sm_mhz": (gu_ms * mhz_prof) if mhz_prof else None,
                      "traffic": (gateup_traffic(cfg.name) if args.layers is None else None), "traffic_unit": "bytes per launch (DRAM read + write, ncu)",
                      "ms_per_launch": gu_ms, "launches_timed": prof["gemm_gateup"][1]},
         "kernels": kernels,
@@ -462,6 +527,22 @@ def run_cascade(args):
     print(json.dumps(out))
 
 
+def replica_command(n: int, argv, port: int):
+    """The launch line for N replicas, one process per GPU: this same file under torch.distributed.run."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+
+
+def spawn_replicas(n: int, argv) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N processes here and hand back their exit status.
+    Rank 0 of the children prints the one JSON line."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    return subprocess.run(replica_command(n, list(argv), port)).returncode
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -470,6 +551,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=2.5,
+                    help="the K-step timed loop is repeated (at least 10 times) until the timed region lasts this long")
     ap.add_argument("--layers", type=int, default=None,
                     help="run a reduced-depth copy of the workload (for profiler captures of single kernels); "
                          "not a benchmark configuration")
@@ -478,6 +561,8 @@ def main():
                          "model runs at that depth)")
     ap.add_argument("--tau", type=float, default=None, help="threshold of the two-tier pass (default: the workload's)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.cascade is None:
+        sys.exit(spawn_replicas(args.gpus, sys.argv[1:]))
     if args.cascade is not None:
         run_cascade(args)
         return

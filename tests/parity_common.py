@@ -87,8 +87,9 @@ def compare(gpu: dict, gpu_logits: Optional[np.ndarray], ref: dict, tau: float, 
 # ordinary row's. The bounds below are not derived from that worst case: they are at most three times the largest
 # error observed on the GPU for the class of model (see the table of observed maxima in the design notes), so a
 # regression of the forward pass by a small factor fails them. Keys: (shallow, deep) = (up to 3 layers, more).
-PLANTED_LOGIT_TOL = {"shallow": 4.5e-2, "deep": 2.4e-1}
-PLANTED_CONF_TOL = {"shallow": 5e-3, "deep": 2.5e-2}
+# Observed worst cases: planted-row logit 2.1e-2 (shallow) / 4.8e-2 (deep), confidence 4.0e-3 / 1.1e-2.
+PLANTED_LOGIT_TOL = {"shallow": 6e-2, "deep": 1.2e-1}
+PLANTED_CONF_TOL = {"shallow": 1e-2, "deep": 3e-2}
 
 
 def planted_tols(cfg):
@@ -139,7 +140,8 @@ def compare_planted(gpu: dict, gpu_logits: np.ndarray, ref: dict, tau: float, cf
     assert stats["planted_logit_err"] <= logit_tol, stats
     assert stats["conf_err"] <= conf_tol, stats
     if gpu_lse is not None:
-        assert stats["lse_err"] <= LOGIT_TOL, stats
+        # where the planted logit dominates the sum, the logsumexp is that logit and moves with it
+        assert stats["lse_err"] <= logit_tol, stats
     assert stats["conf_err_given_logits"] <= 1e-4, stats
     sure = np.abs(conf_z - tau) > 1e-4
     assert np.array_equal(acc[sure], O.gate(conf_z, tau)[sure])

@@ -106,3 +106,24 @@ def test_two_replicas_reduce_times_by_max_and_units_by_sum():
 def test_single_process_aggregation_is_the_identity():
     import bench
     assert bench.aggregate_over_ranks(3.0, 4.0, 16, 1163) == (3.0, 4.0, 16.0, 1163.0)
+
+
+def test_gpus_flag_without_a_launcher_starts_the_replicas():
+    """`python bench.py --gpus 2` started bare must bring up two processes itself. Exercised on the CPU through the
+    oracle-timing arm, whose rank 0 prints the line while the other rank exits without work."""
+    import json
+    import subprocess
+    import bench
+    cmd = bench.replica_command(2, ["--gpus", "2"], 29999)
+    assert "--nproc-per-node=2" in cmd and "127.0.0.1" in cmd and cmd[-2:] == ["--gpus", "2"]
+    env = dict(os.environ)
+    for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK"):
+        env.pop(k, None)
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--workload", "cfg1_tiny", "--steps", "1", "--warmup", "0"],
+                         capture_output=True, text=True, timeout=600, env=env, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                      # one line from rank 0, none from rank 1
+    out = json.loads(lines[0])
+    assert out["impl"] == "reference" and out["n_gpus"] == 2 and out["value"] > 0
