@@ -255,6 +255,8 @@ def run_ours(args, cfg):
         ses.alloc_cache(pages, total, batch.ctx_lens)
         ses.fill_synthetic_context(lambda i, l: context_kv(cfg, i, l, int(batch.ctx_lens[i])))
     B.cs_reserve(ses.model, batch.n_steps, batch.n_tokens)
+    if args.deterministic is not None:
+        B.cs_set_deterministic(ses.model, bool(args.deterministic))
     stream = torch.cuda.current_stream()
     K, W = args.steps, max(3, args.warmup)
     counts = work_counts(cfg, batch)
@@ -409,7 +411,9 @@ def run_ours(args, cfg):
                    "l2": "inputs larger than L2 (3.1 GB of weights streamed every step)",
                    "last_layer": "MLP half on each step's last row only (no other row reaches the LM head); its small "
                                  "launches are timed under 'other', not in the per-launch projection figures",
-                   "replicas": world},
+                   "replicas": world,
+                   "deterministic": ("library default (bit-identical passes)" if args.deterministic is None
+                                     else bool(args.deterministic))},
         "clocks": clocks,
         "clocks_per_kernel_run": clocks_prof,
         "e2e": {"value": all_steps * K / (ms_e2e * 1e-3), "unit": UNIT,
@@ -551,6 +555,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--deterministic", type=int, default=None, choices=[0, 1],
+                    help="cs_set_deterministic for the timed model (default: the library's default, which is 1)")
     ap.add_argument("--min-seconds", type=float, default=2.5,
                     help="the K-step timed loop is repeated (at least 10 times) until the timed region lasts this long")
     ap.add_argument("--layers", type=int, default=None,

@@ -221,8 +221,9 @@ int cs_append_accepted(cs_model* model, cs_kv* kv, int R, const int32_t* req_seq
  *   out_conf           device float[B].
  *   out_accept         device uint8[B]: 1 = the draft decision is trusted, 0 = escalate.
  *   out_verdict        device int32[B] or NULL: index into verdict_ids of the decision r_D.
- * Asynchronous on `stream`. The residual-stream projections accumulate with floating-point atomics, so
- * repeated calls agree to rounding, not bit for bit.
+ * Asynchronous on `stream`. Deterministic: the same call on the same inputs gives bit-identical out_conf, out_accept,
+ * out_verdict (and logits) every time - every reduction of the pass has a fixed order (see cs_set_deterministic).
+ * A model's calls must be issued on one stream at a time: they share its workspace and ordering words.
  * Errors: CS_EINVAL before any launch; CS_ESTATE for an unset sequence; CS_ENOMEM / CS_ECUDA.
  */
 int cs_verify_steps(cs_model* model, const cs_kv* ctx_kv, const int32_t* seq_ids, int B,
@@ -312,6 +313,14 @@ int cs_cascade_select(const uint8_t* trusted, const int32_t* verdict_d, const fl
  * previous query gave up on a bounded wait, else CS_OK.
  */
 int cs_set_keep_logits(cs_model* model, int keep);
+/*
+ * cs_set_deterministic - choose how the residual projections (x += o Wo^T, x += h Wd^T) add the pieces of a long k
+ * range that is cut over several SMs. on != 0 (the default): in a fixed order, one piece of a tile after the other, so
+ * that a pass is bit-identical from run to run - the cascade rule of Eq. 4 is a threshold, and a last-bit difference
+ * in a confidence next to tau would change which steps escalate. on == 0: pieces add as they finish; a little faster,
+ * results agree to rounding only.
+ */
+int cs_set_deterministic(cs_model* model, int on);
 int cs_get_last_logits(cs_model* model, float* dev_out, int B, void* stream);
 int cs_get_last_lse(cs_model* model, float* dev_out, int B, void* stream);
 int cs_last_status(cs_model* model, void* stream);
@@ -334,7 +343,10 @@ int cs_selftest_wait_timeout(cs_model* model, int polls, void* stream);
  */
 /* out[M,N] (+)= a[M,K] * w[N,K]^T on the tcgen05 tensor cores. a, w fp16 row-major (device), fp32 accumulate.
  *   epilogue 0: out fp16 [M,N] = result.
- *   epilogue 1: out fp32 [M,N] += result (atomic adds; split along K over the SMs).
+ *   epilogue 1: out fp32 [M,N] += result. Long k ranges are split over the SMs and the pieces of a tile are added in a
+ *               fixed order (bit-identical from run to run); calls that overlap on the GPU share the ordering words
+ *               and must be kept on one stream.
+ *   epilogue 3: as 1 without the fixed order (pieces add as they finish; results agree to rounding only).
  *   epilogue 2: w2 is a second [N,K] matrix; out fp16 [M,N] = silu(a*w^T) * (a*w2^T).
  * K and N multiples of 8. Asynchronous on `stream`. */
 int cs_gemm_f16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* out,

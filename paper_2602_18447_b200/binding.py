@@ -17,7 +17,7 @@ EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_model_set_lm_head_rows",
     "cs_reserve",
     "cs_kv_alloc", "cs_kv_alloc_8bit", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
-    "cs_verify_steps", "cs_verify_cascade", "cs_append_accepted", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_get_last_logits", "cs_get_last_lse",
+    "cs_verify_steps", "cs_verify_cascade", "cs_append_accepted", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_set_deterministic", "cs_get_last_logits", "cs_get_last_lse",
     "cs_last_status", "cs_selftest_wait_timeout", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
 ]
 
@@ -82,6 +82,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_escalate_mask": (C.c_int, [vp, i32, f32, vp, vp, vp, vp]),
         "cs_cascade_select": (C.c_int, [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]),
         "cs_set_keep_logits": (C.c_int, [vp, i32]),
+        "cs_set_deterministic": (C.c_int, [vp, i32]),
         "cs_get_last_logits": (C.c_int, [vp, vp, i32, vp]),
         "cs_get_last_lse": (C.c_int, [vp, vp, i32, vp]),
         "cs_last_status": (C.c_int, [vp, vp]),
@@ -324,6 +325,10 @@ def cs_cascade_select(trusted, verdict_d, conf_d, verdict_t, conf_t, req_offsets
 
 def cs_set_keep_logits(model: int, keep: bool) -> None:
     _check(load_library().cs_set_keep_logits(model, 1 if keep else 0), "cs_set_keep_logits")
+
+
+def cs_set_deterministic(model: int, on: bool) -> None:
+    _check(load_library().cs_set_deterministic(model, 1 if on else 0), "cs_set_deterministic")
 
 
 def cs_get_last_logits(model: int, out, B: int, stream=None) -> None:

@@ -97,6 +97,10 @@ struct cs_model {
   // workspace
   DevBuf x, x_last, a, qkv, attn_o, hmlp, rope, h_last, lm_part, vlogits, logits, lse, attn_part_o, attn_part_ml, attn_counters;
   uint32_t* status = nullptr;
+  // fixed order of the residual projections' additions (bit-identical passes); see TurnOrder
+  uint32_t* turn_flags = nullptr;
+  uint32_t turn_epoch = 0;
+  bool deterministic = true;
   Staging stg;
   bool keep_logits = false;
   bool last_rows_compact = false;   // the last run_layers left the steps' final hidden rows in x_last, in step order
@@ -413,6 +417,8 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   ap.status = m->status;
   const int plane_groups = kv->num_pages * d.n_kv_heads * kPageSize / 8;
 
+  TurnOrder turn_order{m->turn_flags, &m->turn_epoch};
+  const TurnOrder* turn = m->deterministic ? &turn_order : nullptr;
   RopeEpilogue rope_epi{rope, d.head_dim / 2, (d.n_q_heads + d.n_kv_heads) * d.head_dim};
   rope_epi.q_cols = m->q_dim;
   rope_epi.eps = d.rms_eps;
@@ -448,7 +454,7 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
                                 append_kv->pool + static_cast<size_t>(2 * l + 1) * append_kv->plane_elems,
                                 d.n_kv_heads, d.head_dim, kPageSize, T, 1, s));
     }
-    CS_STEP(kProfO, gemm_f16(tm_o, lw.tm_wo, nullptr, x, T, d.d_model, m->q_dim, kEpiResidAdd, m->status, s));
+    CS_STEP(kProfO, gemm_f16(tm_o, lw.tm_wo, nullptr, x, T, d.d_model, m->q_dim, kEpiResidAdd, m->status, s, turn));
     if (l == d.n_layers - 1 && !append_kv) {
       // Only each step's last position feeds the LM head, and after the last attention no row depends on another:
       // the last MLP runs on those B rows alone. Same arithmetic per row; the launches are small and bound by
@@ -463,13 +469,13 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
       CS_STEP(kProfOther, launch_gather_last_rows(x, dev_meta + L.off_cu, xl, L.B, d.d_model, s));
       CS_STEP(kProfOther, launch_rmsnorm(xl, lw.norm2, a, L.B, d.d_model, d.rms_eps, s));
       CS_STEP(kProfOther, gemm_f16(tm_a_last, lw.tm_wg, &lw.tm_wu, hmlp, L.B, d.d_ffn, d.d_model, kEpiSwiGLU, m->status, s));
-      CS_STEP(kProfOther, gemm_f16(tm_h_last, lw.tm_wd, nullptr, xl, L.B, d.d_model, d.d_ffn, kEpiResidAdd, m->status, s));
+      CS_STEP(kProfOther, gemm_f16(tm_h_last, lw.tm_wd, nullptr, xl, L.B, d.d_model, d.d_ffn, kEpiResidAdd, m->status, s, turn));
       m->last_rows_compact = true;
       break;
     }
     CS_STEP(kProfNorm, launch_rmsnorm(x, lw.norm2, a, T, d.d_model, d.rms_eps, s));
     CS_STEP(kProfGateUp, gemm_f16(tm_a, lw.tm_wg, &lw.tm_wu, hmlp, T, d.d_ffn, d.d_model, kEpiSwiGLU, m->status, s));
-    CS_STEP(kProfDown, gemm_f16(tm_h, lw.tm_wd, nullptr, x, T, d.d_model, d.d_ffn, kEpiResidAdd, m->status, s));
+    CS_STEP(kProfDown, gemm_f16(tm_h, lw.tm_wd, nullptr, x, T, d.d_model, d.d_ffn, kEpiResidAdd, m->status, s, turn));
   }
   return CS_OK;
 }
@@ -579,6 +585,8 @@ int stage_batch(cs_model* m, const cs_kv* kv, const int32_t* seq_ids, int B, con
 }
 
 uint32_t* g_test_status = nullptr;
+uint32_t* g_test_turn_flags = nullptr;
+uint32_t g_test_turn_epoch = 0;
 
 }  // namespace
 
@@ -716,6 +724,12 @@ int cs_model_load(const cs_model_desc* desc, const cs_model_tensors* t, int on_d
     m->owned.push_back(p);
     m->status = static_cast<uint32_t*>(p);
     cudaMemset(p, 0, 256);
+    p = nullptr;
+    e = cudaMalloc(&p, sizeof(uint32_t) * kTurnWords);
+    if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc(turn flags)"); cs_model_free(m); return rc; }
+    m->owned.push_back(p);
+    m->turn_flags = static_cast<uint32_t*>(p);
+    cudaMemset(p, 0, sizeof(uint32_t) * kTurnWords);
   }
 #undef CS_TRY
   CS_CUDA(cudaDeviceSynchronize());
@@ -1136,6 +1150,12 @@ int cs_cascade_select(const uint8_t* trusted, const int32_t* verdict_d, const fl
 
 int64_t cs_last_h2d_bytes(const cs_model* m) { return m ? m->last_h2d_bytes : 0; }
 
+int cs_set_deterministic(cs_model* m, int on) {
+  if (!m) return CS_EINVAL;
+  m->deterministic = on != 0;
+  return CS_OK;
+}
+
 int cs_set_keep_logits(cs_model* m, int keep) {
   if (!m) return CS_EINVAL;
   m->keep_logits = keep != 0;
@@ -1206,7 +1226,7 @@ int cs_profile_read(cs_model* m, float* ms_out, int32_t* launches_out, int n_cla
 
 int cs_gemm_f16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* out, int M, int N, int K,
                  int epilogue, void* stream) {
-  if (!a || !w || !out || M < 0 || N < 8 || K < 8 || (N % 8) || (K % 8) || epilogue < 0 || epilogue > 2)
+  if (!a || !w || !out || M < 0 || N < 8 || K < 8 || (N % 8) || (K % 8) || epilogue < 0 || epilogue > 3)
     return CS_EINVAL;
   if (epilogue == kEpiSwiGLU && !w2) return CS_EINVAL;
   if (M == 0) return CS_OK;
@@ -1220,8 +1240,13 @@ int cs_gemm_f16(const uint16_t* a, const uint16_t* w, const uint16_t* w2, void* 
     g_cuda_error = "cuTensorMapEncodeTiled failed";
     return CS_ECUDA;
   }
-  CS_CUDA(gemm_f16(ta, tb, w2 ? &tb2 : nullptr, out, M, N, K, epilogue, g_test_status,
-                    static_cast<cudaStream_t>(stream)));
+  if (!g_test_turn_flags) {
+    CS_CUDA(cudaMalloc(reinterpret_cast<void**>(&g_test_turn_flags), sizeof(uint32_t) * kTurnWords));
+    CS_CUDA(cudaMemset(g_test_turn_flags, 0, sizeof(uint32_t) * kTurnWords));
+  }
+  TurnOrder turn{g_test_turn_flags, &g_test_turn_epoch};
+  CS_CUDA(gemm_f16(ta, tb, w2 ? &tb2 : nullptr, out, M, N, K, epilogue == 3 ? kEpiResidAdd : epilogue, g_test_status,
+                    static_cast<cudaStream_t>(stream), epilogue == 1 ? &turn : nullptr));
   return CS_OK;
 }
 

@@ -9,7 +9,7 @@ namespace cs {
 
 enum GemmEpilogue {
   kEpiStoreF16 = 0,  // out fp16 [M,N] = a * w^T
-  kEpiResidAdd = 1,   // out fp32 [M,N] += a * w^T   (atomic adds, k-range split over the SMs)
+  kEpiResidAdd = 1,   // out fp32 [M,N] += a * w^T   (added by the copy engine; long k ranges are split over the SMs)
   kEpiSwiGLU = 2,     // out fp16 [M,N] = silu(a * w^T) * (a * w2^T)
   kEpiStoreRope = 3,  // out fp16 [M,N] = a * w^T with the rotary turn applied to the leading heads (QKV projection)
   kEpiStoreNormRope = 4   // as kEpiStoreRope, each turned head RMS-normalised over its columns first (gains qk_gain)
@@ -56,7 +56,16 @@ struct RopeEpilogue {
 cudaError_t gemm_f16_rope(const CUtensorMap& ta, const CUtensorMap& tb, void* out, int M, int N, int K,
                           const RopeEpilogue& rope, uint32_t* status, cudaStream_t stream);
 
+// Ordered mode of the residual epilogue (kEpiResidAdd): `flags` is a zero-initialised device array of
+// kTurnWords words that only these launches touch, `epoch` a host counter that every ordered launch advances. With it the pieces
+// of a tile are added in a fixed order and the result is bit-identical from run to run; launches that share the array
+// must be ordered on one stream.
+constexpr int kTurnWords = 148 + 8;
+struct TurnOrder {
+  uint32_t* flags;
+  uint32_t* epoch;
+};
 cudaError_t gemm_f16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,
-                      int K, int epilogue, uint32_t* status, cudaStream_t stream);
+                      int K, int epilogue, uint32_t* status, cudaStream_t stream, const TurnOrder* turn = nullptr);
 
 }  // namespace cs

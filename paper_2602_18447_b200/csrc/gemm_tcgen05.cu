@@ -9,7 +9,13 @@
 // sum (fp16 store, SwiGLU) the ranges are whole tiles. For the residual epilogue (x += a * w^T, fp32) the
 // range is cut evenly over the SMs whatever the tile boundaries are, and every piece is added into x by the copy
 // engine (TMA reduce-add from a shared-memory box), which is what lets the narrow O and down projections fill all SMs.
+// The pieces of one tile belong to consecutive CTAs. In the ordered mode they add in a fixed order - the piece with the
+// highest k range first, which is also the one that finishes first - so that every element of x receives its pieces
+// in the same order in every run and the result is bit-identical from run to run: a piece waits (bounded) for a word
+// that the CTA holding the next k range of its tile sets once its own additions have been performed.
 #include "gemm.h"
+
+#include <algorithm>
 
 #include "kernels.h"
 
@@ -23,6 +29,8 @@ constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int kGemmThreads = 192;
 constexpr int kABytes = BM * BK * 2;
+constexpr int kMaxOrderedPieces = 4;    // ordered residual epilogue: a tile's k range is cut into about this many pieces at most
+constexpr int kShortK = 2048;           // residual projections with K up to this run on whole 128-wide tiles
 
 template <int BN>
 struct GemmSmem {
@@ -41,11 +49,52 @@ struct Segment {
   int tile, kb0, len;
 };
 
-__device__ __forceinline__ Segment next_segment(int u, int end, int kblocks) {
+// A CTA's range of k-blocks [start, end) as a sequence of segments. A range may begin inside a tile (a "head" piece
+// up to that tile's end, or a "middle" piece if the whole range lies inside the tile) and may stop short of a tile's
+// end (a "tail" piece, which begins at its tile's start). The pieces come first, the whole tiles after them: what other
+// CTAs wait for (ordered residual epilogue) is finished early, and a CTA ends on a tile that it shares with nobody.
+struct SegPlan {
+  int start, kblocks, head_len, tail_len, whole0, n_whole, count;
+};
+__device__ __forceinline__ SegPlan make_plan(int start, int end, int kblocks) {
+  SegPlan p;
+  p.start = start;
+  p.kblocks = kblocks;
+  p.head_len = p.tail_len = p.n_whole = p.count = 0;
+  p.whole0 = start;
+  if (start >= end) return p;
+  const int r = start % kblocks;
+  if (r != 0) p.head_len = min(kblocks - r, end - start);
+  p.whole0 = start + p.head_len;
+  const int rem = end - p.whole0;
+  p.n_whole = rem / kblocks;
+  p.tail_len = rem - p.n_whole * kblocks;
+  p.count = (p.head_len > 0) + (p.tail_len > 0) + p.n_whole;
+  return p;
+}
+__device__ __forceinline__ Segment plan_segment(const SegPlan& p, int i) {
   Segment s;
-  s.tile = u / kblocks;
-  s.kb0 = u - s.tile * kblocks;
-  s.len = min(kblocks - s.kb0, end - u);
+  if (p.head_len > 0) {
+    if (i == 0) {
+      s.tile = p.start / p.kblocks;
+      s.kb0 = p.start - s.tile * p.kblocks;
+      s.len = p.head_len;
+      return s;
+    }
+    --i;
+  }
+  if (p.tail_len > 0) {
+    if (i == 0) {
+      s.tile = p.whole0 / p.kblocks + p.n_whole;
+      s.kb0 = 0;
+      s.len = p.tail_len;
+      return s;
+    }
+    --i;
+  }
+  s.tile = p.whole0 / p.kblocks + i;
+  s.kb0 = 0;
+  s.len = p.kblocks;
   return s;
 }
 
@@ -74,6 +123,30 @@ __device__ __forceinline__ void bulk_wait_group_read() {
   asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Ordered mode of the residual epilogue. The pieces of a tile belong to consecutive CTAs and add in descending order
+// of their k range: head, middle pieces, tail. Every CTA owns one word, which it sets to the launch's number once the
+// additions of the piece at the start of its range (head or middle) have been performed; a middle or tail piece waits
+// (bounded) for the word of the CTA above it. A head piece is the first thing its CTA computes, so in launches whose
+// CTAs each hold more than a tile nobody ever waits long.
+constexpr uint32_t kTurnSpinLimit = 1u << 22;     // polls of ~0.1-0.3 us each: about a second
+__device__ __forceinline__ bool wait_turn(const uint32_t* flag, uint32_t epoch, volatile uint32_t* abort_flag,
+                                          uint32_t* status) {
+  for (uint32_t i = 0; i < kTurnSpinLimit; ++i) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v == epoch) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+    __nanosleep(i < 64 ? 32 : 256);
+  }
+  *abort_flag = 1;
+  atomicOr(status, kStatusTimeout);
+  return false;
+}
+__device__ __forceinline__ void publish_turn(uint32_t* flag, uint32_t epoch) {
+  asm volatile("fence.proxy.async;" ::: "memory");     // the additions went through the copy engine
+  __threadfence();
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(epoch) : "memory");
+}
 __device__ __forceinline__ void st_shared_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(p)), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -125,7 +198,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                  const __grid_constant__ CUtensorMap tm_b2, const __grid_constant__ CUtensorMap tm_out,
                  void* __restrict__ out, int M, int N, int m_tiles, int n_tiles, int kblocks, int total_units,
-                 int units_per_cta, const RopeEpilogue rope, uint32_t* status) {
+                 int units_per_cta, const RopeEpilogue rope, uint32_t* status, uint32_t* turn_flags, uint32_t epoch) {
   using L = GemmSmem<BN>;
   constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
   constexpr uint32_t kTmemCols = 2 * BN;
@@ -138,7 +211,8 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   uint64_t* empty_bar = bars + L::kStages;         // [kStages] MMA -> TMA
   uint64_t* acc_full = bars + 2 * L::kStages;      // [2] MMA -> epilogue
   uint64_t* acc_empty = bars + 2 * L::kStages + 2; // [2] epilogue -> MMA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * L::kStages + 4);
+  uint64_t* turn_bar = bars + 2 * L::kStages + 4;  // the epilogue warps' additions of the first piece are done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * L::kStages + 5);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5;
@@ -146,6 +220,7 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
   const int start = blockIdx.x * units_per_cta;
   const int end = min(total_units, start + units_per_cta);
+  const SegPlan plan = make_plan(start, end, kblocks);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < L::kStages; ++s) {
@@ -156,6 +231,7 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       mbar_init(&acc_full[a], 1);
       mbar_init(&acc_empty[a], 4);
     }
+    mbar_init(turn_bar, 4);
     *abort_flag = 0;
     fence_barrier_init();
     tma_prefetch_desc(&tm_a);
@@ -174,16 +250,18 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   pdl_launch_dependents();
   // The producer thread waits a little later: the weights do not depend on the previous kernel, so it first sends
   // for the B boxes of its first stages (all stages are empty at this point).
-  const int pre = (threadIdx.x == 0) ? max(0, min(L::kStages, end - start)) : 0;
+  int pre = 0;
   if (threadIdx.x == 0) {
-    for (int i = 0; i < pre; ++i) {
-      const int u = start + i, tile = u / kblocks, kb = u - tile * kblocks;
-      const int n0 = tile_n(tile, m_tiles, n_tiles, EPI) * OUT_BN;
-      uint8_t* sb = smem + i * L::kStageBytes + kABytes;
-      mbar_arrive_expect_tx(&full_bar[i], L::kStageBytes);
-      tma_load_2d(sb, &tm_b, &full_bar[i], kb * BK, n0);
-      if (EPI == kEpiSwiGLU) tma_load_2d(sb + 128 * BK * 2, &tm_b2, &full_bar[i], kb * BK, n0);
-      else if (BN == 256) tma_load_2d(sb + 128 * BK * 2, &tm_b, &full_bar[i], kb * BK, n0 + 128);
+    for (int si = 0; si < plan.count && pre < L::kStages; ++si) {
+      const Segment sg = plan_segment(plan, si);
+      const int n0 = tile_n(sg.tile, m_tiles, n_tiles, EPI) * OUT_BN;
+      for (int kb = sg.kb0; kb < sg.kb0 + sg.len && pre < L::kStages; ++kb, ++pre) {
+        uint8_t* sb = smem + pre * L::kStageBytes + kABytes;
+        mbar_arrive_expect_tx(&full_bar[pre], L::kStageBytes);
+        tma_load_2d(sb, &tm_b, &full_bar[pre], kb * BK, n0);
+        if (EPI == kEpiSwiGLU) tma_load_2d(sb + 128 * BK * 2, &tm_b2, &full_bar[pre], kb * BK, n0);
+        else if (BN == 256) tma_load_2d(sb + 128 * BK * 2, &tm_b, &full_bar[pre], kb * BK, n0 + 128);
+      }
     }
   }
   pdl_wait();
@@ -196,8 +274,8 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int u = start; u < end && ok;) {
-        const Segment sg = next_segment(u, end, kblocks);
+      for (int si = 0; si < plan.count && ok; ++si) {
+        const Segment sg = plan_segment(plan, si);
         const int m0 = tile_m(sg.tile, m_tiles, n_tiles, EPI) * BM;
         const int n0 = tile_n(sg.tile, m_tiles, n_tiles, EPI) * OUT_BN;
         for (int kb = sg.kb0; kb < sg.kb0 + sg.len; ++kb, ++issued) {
@@ -216,7 +294,6 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           }
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
-        u += sg.len;
       }
       // In a healthy run the MMA warp has waited for every copy before the CTA exits. After an abort, give
       // the copies still in flight time to land in shared memory before the CTA may go away.
@@ -238,8 +315,8 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       const uint64_t adesc0 = umma_desc_k128(smem_base);
       const uint64_t bdesc0 = umma_desc_k128(smem_base + kABytes);
       bool ready = false;
-      for (int u = start; u < end && ok;) {
-        const Segment sg = next_segment(u, end, kblocks);
+      for (int si = 0; si < plan.count && ok; ++si) {
+        const Segment sg = plan_segment(plan, si);
         if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
@@ -256,7 +333,6 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         umma_commit(&acc_full[acc]);
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
-        u += sg.len;
       }
     }
   } else {
@@ -265,8 +341,10 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int u = start; u < end && ok;) {
-      const Segment sg = next_segment(u, end, kblocks);
+    const bool ordered = EPI == kEpiResidAdd && turn_flags != nullptr;
+    bool owes_turn = ordered && plan.head_len > 0;
+    for (int si = 0; si < plan.count && ok; ++si) {
+      const Segment sg = plan_segment(plan, si);
       const int m0 = tile_m(sg.tile, m_tiles, n_tiles, EPI) * BM;
       const int n0 = tile_n(sg.tile, m_tiles, n_tiles, EPI) * OUT_BN;
       const int row = m0 + quad * 32 + lane;
@@ -399,6 +477,15 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // main loop. Two boxes per warp alternate; lane 0 owns the warp's copy groups.
         uint8_t* stage0 = smem + L::kStagingOff + quad * 2 * 4096;
         const int y = m0 + quad * 32;
+        // Ordered mode: a piece that stops short of its tile's end adds after the piece above it (next CTA); a piece
+        // that starts inside its tile tells the piece below it (previous CTA) when its own additions are done.
+        const bool partial = ordered && sg.len < kblocks;
+        const bool publishes = partial && sg.kb0 > 0;
+        const int me = blockIdx.x;
+        if (partial && sg.kb0 + sg.len < kblocks) {
+          if (!wait_turn(turn_flags + me + 1, epoch, abort_flag, status)) { ok = false; break; }
+          asm volatile("fence.proxy.async;" ::: "memory");
+        }
 #pragma unroll 1
         for (int c = 0; c < BN / 32 && n0 + c * 32 < N; ++c) {
           tmem_ld_32x32(t_row + c * 32, r);
@@ -420,15 +507,27 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
         if (lane == 0) bulk_wait_group_read<0>();
         __syncwarp();
+        if (publishes) {
+          // additions performed by all four warps -> the piece below may add
+          if (lane == 0) {
+            bulk_wait_group_all();
+            mbar_arrive(turn_bar);
+          }
+          if (warp == 2 && lane == 0 && mbar_wait(turn_bar, 0, abort_flag, status)) {
+            publish_turn(turn_flags + me, epoch);
+            owes_turn = false;
+          }
+        }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
-      u += sg.len;
     }
     if (EPI == kEpiResidAdd && lane == 0) bulk_wait_group_all();   // the additions have been performed
+    // A CTA that gave up still lets the pieces that wait for it go on (the time-out is reported through the status word).
+    if (owes_turn && warp == 2 && lane == 0) publish_turn(turn_flags + blockIdx.x, epoch);
   }
 
   tc_fence_before();
@@ -469,7 +568,8 @@ bool make_out_f32_map(CUtensorMap* tm, void* base, int rows, int cols) {
 
 template <int BN, int EPI>
 cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, void* out, int M, int N,
-                   int K, uint32_t* status, cudaStream_t stream, const RopeEpilogue& rope = RopeEpilogue{nullptr, 0, 0}) {
+                   int K, uint32_t* status, cudaStream_t stream, const RopeEpilogue& rope = RopeEpilogue{nullptr, 0, 0},
+                   const TurnOrder* turn = nullptr, bool whole_tiles = false) {
   using L = GemmSmem<BN>;
   constexpr int OUT_BN = (EPI == kEpiSwiGLU) ? BN / 2 : BN;
   static std::atomic<uint64_t> smem_opted{0};
@@ -480,9 +580,18 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
   const int tiles = m_tiles * n_tiles;
   const int total = tiles * kblocks;
   int grid, upc;
-  if (EPI == kEpiResidAdd) {
+  uint32_t* turn_flags = nullptr;
+  uint32_t epoch = 0;
+  if (EPI == kEpiResidAdd && !whole_tiles) {
     grid = total < kNumSMs ? total : kNumSMs;
     upc = (total + grid - 1) / grid;
+    if (turn) {
+      // The pieces of a tile add one after the other: keep them few when the even cut would make them many (few rows).
+      upc = std::max(upc, (kblocks + kMaxOrderedPieces - 1) / kMaxOrderedPieces);
+      turn_flags = turn->flags;
+      epoch = ++*turn->epoch;
+      if (epoch == 0) epoch = ++*turn->epoch;       // 0 is what a fresh flag array holds
+    }
     grid = (total + upc - 1) / upc;
   } else {
     const int tpc = (tiles + kNumSMs - 1) / kNumSMs;
@@ -492,7 +601,7 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
   CUtensorMap tout = ta;   // only the residual epilogue reads it
   if (EPI == kEpiResidAdd && !make_out_f32_map(&tout, out, M, N)) return cudaErrorInvalidValue;
   cudaError_t le = launch_pdl(gemm_f16_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), L::kTotal, stream, ta, tb, tb2, tout, out, M,
-                              N, m_tiles, n_tiles, kblocks, total, upc, rope, status);
+                              N, m_tiles, n_tiles, kblocks, total, upc, rope, status, turn_flags, epoch);
   count_launch();
   return le != cudaSuccess ? le : cudaGetLastError();
 }
@@ -571,7 +680,7 @@ cudaError_t gemm_f16_rope(const CUtensorMap& ta, const CUtensorMap& tb, void* ou
 }
 
 cudaError_t gemm_f16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap* tb2, void* out, int M, int N,
-                      int K, int epilogue, uint32_t* status, cudaStream_t stream) {
+                      int K, int epilogue, uint32_t* status, cudaStream_t stream, const TurnOrder* turn) {
   if (M <= 0) return cudaSuccess;
   switch (epilogue) {
     case kEpiStoreF16:
@@ -580,7 +689,11 @@ cudaError_t gemm_f16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtenso
       if (N <= 128) return launch<128, kEpiStoreF16>(ta, tb, tb, out, M, N, K, status, stream);
       return launch<256, kEpiStoreF16>(ta, tb, tb, out, M, N, K, status, stream);
     case kEpiResidAdd:
-      return launch<256, kEpiResidAdd>(ta, tb, tb, out, M, N, K, status, stream);
+      // Short k ranges (the O projection): whole 128-wide tiles. The narrow tiles are issue-bound, but there are twice
+      // as many of them, no tile is shared between CTAs and every element of the output receives one addition.
+      if (K <= kShortK && N >= 128)
+        return launch<128, kEpiResidAdd>(ta, tb, tb, out, M, N, K, status, stream, RopeEpilogue{nullptr, 0, 0}, nullptr, true);
+      return launch<256, kEpiResidAdd>(ta, tb, tb, out, M, N, K, status, stream, RopeEpilogue{nullptr, 0, 0}, turn);
     case kEpiSwiGLU:
       return launch<256, kEpiSwiGLU>(ta, tb, *tb2, out, M, N, K, status, stream);
     default:

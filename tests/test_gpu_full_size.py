@@ -51,6 +51,12 @@ def _run_full(name, weights, n_sample, always=()):
         vid = list(cfg.verdict_ids)
         assert np.max(np.abs(np.exp(z[:, vid] - lse_from_logits[:, None]).max(axis=1) - gpu["conf"])) < 1e-6
         del z
+        # the pass is deterministic: a second run gives the same bits (logits of all steps, confidences, mask)
+        ses.verify()
+        again = ses.results()
+        assert np.array_equal(again["conf"].view(np.uint32), gpu["conf"].view(np.uint32))
+        assert np.array_equal(again["accept"], gpu["accept"]) and np.array_equal(again["verdict"], gpu["verdict"])
+        assert np.array_equal(ses.last_logits().view(np.uint32), logits.view(np.uint32))
 
         # ---- planted verdict rows, same session
         wp, ids, rows = _planted_rows(cfg, weights)
