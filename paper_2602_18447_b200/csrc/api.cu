@@ -1015,8 +1015,8 @@ int cs_verify_steps(cs_model* m, const cs_kv* ckv, const int32_t* seq_ids, int B
   else
     CS_STEP(kProfNorm, launch_last_rows_norm(x, dev_meta + L.off_cu, m->final_norm, h_last, B, B_all, d.d_model, d.rms_eps, s));
   CUtensorMap tm_h;
-  int tiles_per_cta;
-  const int grid = lm_head_grid(d.vocab, &tiles_per_cta);
+  int rows_per_cta;
+  const int grid = lm_head_grid(d.vocab, &rows_per_cta);
   for (int b0 = 0; b0 < B; b0 += 64) {
     const int bc = std::min(64, B - b0);
     const int bp = lm_head_batch_pad(bc);
@@ -1277,8 +1277,8 @@ int cs_lm_head_gate(const uint16_t* w_lm, const uint16_t* h, int B, int d_model,
     g_cuda_error = "cuTensorMapEncodeTiled failed for the LM head";
     return CS_ECUDA;
   }
-  int tiles_per_cta;
-  const int grid = lm_head_grid(vocab, &tiles_per_cta);
+  int rows_per_cta;
+  const int grid = lm_head_grid(vocab, &rows_per_cta);
   for (int b0 = 0; b0 < B; b0 += 64) {
     const int bc = std::min(64, B - b0);
     const int bp = lm_head_batch_pad(bc);

@@ -26,10 +26,11 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const uint16_t*
   }
 }
 
-// One warp per row. Rows of up to 4096 values are held in registers between the sum of squares and the scaling, so
-// x is read once and all of a row's loads are in flight together; longer rows are read twice.
-constexpr int kNormRegVecs = 32;   // float4 per lane
-
+// One warp per row. A row of up to 128 NV values is held in registers between the sum of squares and the scaling, so x
+// is read once and all of a row's loads are in flight together; longer rows are read twice. The gains are requested
+// together with the row (while they fit the register file): the kernel moves a few MB and lasts as long as its
+// longest chain of dependent memory accesses.
+template <int NV>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
                                uint16_t* __restrict__ out, int rows, int d, float eps) {
   pdl_launch_dependents();
@@ -41,24 +42,32 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
   const float4* g4 = reinterpret_cast<const float4*>(gain);
   uint2* o = reinterpret_cast<uint2*>(out + static_cast<size_t>(row) * d);
   const int n = d >> 2;
-  if (n <= 32 * kNormRegVecs) {
-    float4 v[kNormRegVecs];
+  if (n <= 32 * NV) {
+    constexpr bool kGainsAhead = NV <= 16;
+    float4 v[NV], gv[kGainsAhead ? NV : 1];
     float ss = 0.f;
 #pragma unroll
-    for (int i = 0; i < kNormRegVecs; ++i) {
+    for (int i = 0; i < NV; ++i) {
       const int idx = lane + 32 * i;
       if (idx < n) v[i] = xr[idx];
     }
+    if (kGainsAhead) {
 #pragma unroll
-    for (int i = 0; i < kNormRegVecs; ++i)
+      for (int i = 0; i < NV; ++i) {
+        const int idx = lane + 32 * i;
+        if (idx < n) gv[kGainsAhead ? i : 0] = __ldg(g4 + idx);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < NV; ++i)
       if (lane + 32 * i < n) ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
     ss = warp_sum(ss);
     const float r = rsqrtf(ss / static_cast<float>(d) + eps);
 #pragma unroll
-    for (int i = 0; i < kNormRegVecs; ++i) {
+    for (int i = 0; i < NV; ++i) {
       const int idx = lane + 32 * i;
       if (idx < n) {
-        const float4 g = g4[idx];
+        const float4 g = kGainsAhead ? gv[kGainsAhead ? i : 0] : __ldg(g4 + idx);
         o[idx] = make_uint2(pack_f16x2(v[i].x * r * g.x, v[i].y * r * g.y), pack_f16x2(v[i].z * r * g.z, v[i].w * r * g.w));
       }
     }
@@ -204,7 +213,11 @@ cudaError_t launch_rmsnorm(const float* x, const float* gain, uint16_t* out, int
                            cudaStream_t s) {
   if (rows <= 0) return cudaSuccess;
   const int warps = 4;
-  cudaError_t le = launch_pdl(rmsnorm_kernel, dim3((rows + warps - 1) / warps), dim3(warps * 32), 0, s, x, gain, out, rows, d, eps);
+  const dim3 grid((rows + warps - 1) / warps), block(warps * 32);
+  cudaError_t le;
+  if (d <= 1024) le = launch_pdl(rmsnorm_kernel<8>, grid, block, 0, s, x, gain, out, rows, d, eps);
+  else if (d <= 2048) le = launch_pdl(rmsnorm_kernel<16>, grid, block, 0, s, x, gain, out, rows, d, eps);
+  else le = launch_pdl(rmsnorm_kernel<32>, grid, block, 0, s, x, gain, out, rows, d, eps);
   count_launch();
   return le != cudaSuccess ? le : cudaGetLastError();
 }

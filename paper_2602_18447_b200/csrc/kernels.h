@@ -111,7 +111,8 @@ cudaError_t launch_lm_head(const CUtensorMap& tm_w, const CUtensorMap& tm_h, int
                            int vocab, const int32_t* verdict_ids_host, int n_verdict, float* part_max,
                            float* part_sum, float* verdict_logits, float* logits_or_null, uint32_t* status,
                            cudaStream_t s);
-int lm_head_grid(int vocab, int* tiles_per_cta);
+// Grid of the LM-head launch: the vocabulary is cut evenly into one range of rows per CTA.
+int lm_head_grid(int vocab, int* rows_per_cta);
 int lm_head_batch_pad(int B);
 // Merge the CTAs' pairs, form the confidence and apply the threshold.
 cudaError_t launch_gate(const float* part_max, const float* part_sum, int n_slices, int nb_stride,

@@ -40,8 +40,40 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16])
       : "memory");
 }
 
+// One 64-deep block of products (four K = 16 steps; the descriptors advance by 32 bytes per step), then an arrival on
+// `commit_bar` once they have completed. Before them a non-blocking test of `peek_bar` is issued; its answer (1 = that
+// phase is complete) is read after everything else has been issued: with at most 64 steps per pass the products are
+// short, and a blocking wait between them would leave the tensor core idle for longer than they run.
+__device__ __forceinline__ bool lm_kblock_peek(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate_first, uint64_t* commit_bar, uint64_t* peek_bar,
+                                               uint32_t peek_parity) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred P, Q;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "setp.ne.b32 Q, %7, 0;\n\t"
+      "add.u64 a1, %4, 2;\n\tadd.u64 b1, %5, 2;\n\t"
+      "add.u64 a2, %4, 4;\n\tadd.u64 b2, %5, 4;\n\t"
+      "add.u64 a3, %4, 6;\n\tadd.u64 b3, %5, 6;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, Q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], a1, b1, %6, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], a2, b2, %6, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], a3, b3, %6, 1;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ready)
+      : "r"(smem_u32(peek_bar)), "r"(peek_parity), "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc),
+        "r"(accumulate_first), "r"(smem_u32(commit_bar))
+      : "memory");
+  return ready != 0;
+}
+
+// Rows of the vocabulary [blockIdx.x * rows_per_cta, + rows_per_cta) belong to a CTA, cut evenly so that every SM
+// streams the same number of bytes. A range is walked in 128-row tiles; when it is not a multiple of 128 its last,
+// partial tile comes FIRST: the rows that tile fetches beyond the range are the first tile of the next CTA, which
+// fetches them at the same moment, so they cross the DRAM interface once.
 struct LmArgs {
-  int B, vocab, kblocks, n_tiles, tiles_per_cta, n_verdict, h_row0;
+  int B, vocab, kblocks, rows_per_cta, n_verdict, h_row0;
   int verdict[kLmMaxVerdict];
   float* part_max;        // [grid, NB]
   float* part_sum;        // [grid, NB]
@@ -69,8 +101,15 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   float* red = reinterpret_cast<float*>(smem + L::kRedOff);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile_begin = blockIdx.x * a.tiles_per_cta;
-  const int tile_end = min(a.n_tiles, tile_begin + a.tiles_per_cta);
+  const int row_begin = blockIdx.x * a.rows_per_cta;
+  const int row_end = min(a.vocab, row_begin + a.rows_per_cta);
+  const int n_my_tiles = (row_end - row_begin + kLmBM - 1) / kLmBM;
+  const bool tail_first = ((row_end - row_begin) % kLmBM) != 0 && n_my_tiles > 1;
+  // first row of the i-th tile this CTA works on
+  auto tile_row0 = [&](int i) {
+    const int t = tail_first ? (i == 0 ? n_my_tiles - 1 : i - 1) : i;
+    return row_begin + t * kLmBM;
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < L::kStages; ++s) {
@@ -102,12 +141,13 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int t = tile_begin; t < tile_end && ok; ++t) {
+      for (int i = 0; i < n_my_tiles && ok; ++i) {
+        const int r0 = tile_row0(i);
         for (int kb = 0; kb < a.kblocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, a.status)) { ok = false; break; }
           uint8_t* sw = smem + stage * L::kStageBytes;
           mbar_arrive_expect_tx(&full_bar[stage], kLmWBytes + L::kHBytes);
-          tma_load_2d(sw, &tm_w, &full_bar[stage], kb * kLmBK, t * kLmBM);
+          tma_load_2d(sw, &tm_w, &full_bar[stage], kb * kLmBK, r0);
           tma_load_2d(sw + kLmWBytes, &tm_h, &full_bar[stage], kb * kLmBK, a.h_row0);
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
@@ -119,22 +159,22 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     if (lane == 0) {
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
-      bool ok = true;
-      for (int t = tile_begin; t < tile_end && ok; ++t) {
+      bool ok = true, ready = false;
+      const uint32_t smem_base = smem_u32(smem);
+      const uint64_t adesc0 = umma_desc_k128(smem_base);
+      const uint64_t bdesc0 = umma_desc_k128(smem_base + kLmWBytes);
+      for (int i = 0; i < n_my_tiles && ok; ++i) {
         if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * NB;
         for (int kb = 0; kb < a.kblocks; ++kb) {
-          if (!mbar_wait(&full_bar[stage], phase, abort_flag, a.status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t sw = smem_u32(smem + stage * L::kStageBytes);
-          const uint64_t adesc = umma_desc_k128(sw);
-          const uint64_t bdesc = umma_desc_k128(sw + kLmWBytes);
-#pragma unroll
-          for (int k = 0; k < kLmBK / 16; ++k)
-            umma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0);
-          umma_commit(&empty_bar[stage]);
-          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+          if (!ready && !mbar_wait(&full_bar[stage], phase, abort_flag, a.status)) { ok = false; break; }
+          const int ns = (stage + 1 == L::kStages) ? 0 : stage + 1;
+          const uint32_t np = (ns == 0) ? phase ^ 1u : phase;
+          const uint64_t off = static_cast<uint64_t>(stage * (L::kStageBytes >> 4));
+          ready = lm_kblock_peek(d_tmem, adesc0 + off, bdesc0 + off, kIdesc, kb != 0, &empty_bar[stage], &full_bar[ns], np);
+          stage = ns;
+          phase = np;
         }
         if (!ok) break;
         umma_commit(&acc_full[acc]);
@@ -150,12 +190,12 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int t = tile_begin; t < tile_end; ++t) {
+    for (int i = 0; i < n_my_tiles; ++i) {
       if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, a.status)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + acc * NB + (static_cast<uint32_t>(quad * 32) << 16);
-      const int row = t * kLmBM + quad * 32 + lane;   // vocabulary id of this thread's lane
-      const bool row_ok = row < a.vocab;
+      const int row = tile_row0(i) + quad * 32 + lane;   // vocabulary id of this thread's lane
+      const bool row_ok = row < row_end;                 // rows past the range belong to the next CTA (or to nobody)
       uint32_t vmask = 0;   // which entries of verdict_ids name this row (an id may be listed twice)
       for (int j = 0; j < a.n_verdict; ++j)
         if (a.verdict[j] == row) vmask |= 1u << j;
@@ -442,11 +482,12 @@ cudaError_t launch_lm_nb(const CUtensorMap& tm_w, const CUtensorMap& tm_h, const
 
 }  // namespace
 
-int lm_head_grid(int vocab, int* tiles_per_cta) {
+int lm_head_grid(int vocab, int* rows_per_cta) {
   const int n_tiles = (vocab + kLmBM - 1) / kLmBM;
-  const int tpc = (n_tiles + kNumSMs - 1) / kNumSMs;
-  *tiles_per_cta = tpc;
-  return (n_tiles + tpc - 1) / tpc;
+  const int ctas = n_tiles < kNumSMs ? n_tiles : kNumSMs;
+  const int rows = (vocab + ctas - 1) / ctas;
+  *rows_per_cta = rows;
+  return (vocab + rows - 1) / rows;
 }
 
 int lm_head_batch_pad(int B) { return B <= 16 ? 16 : (B <= 32 ? 32 : 64); }
@@ -460,8 +501,7 @@ cudaError_t launch_lm_head(const CUtensorMap& tm_w, const CUtensorMap& tm_h, int
   a.h_row0 = h_row0;
   a.vocab = vocab;
   a.kblocks = (d + kLmBK - 1) / kLmBK;
-  a.n_tiles = (vocab + kLmBM - 1) / kLmBM;
-  const int grid = lm_head_grid(vocab, &a.tiles_per_cta);
+  const int grid = lm_head_grid(vocab, &a.rows_per_cta);
   a.n_verdict = n_verdict;
   for (int j = 0; j < kLmMaxVerdict; ++j) a.verdict[j] = j < n_verdict ? verdict_ids_host[j] : -1;
   a.part_max = part_max;
@@ -613,8 +653,8 @@ extern "C" int cs_lm_head_gate_static(const uint16_t* w_lm, const uint16_t* h, i
   if (!make_gemm_operand_map(&tm_w, w_lm, vocab, d_model) ||
       !make_tensor_map_16b(&tm_h, h, B, d_model, bp, 64, true, false))      // rows past B read as zeros
     return CS_ECUDA;
-  int tiles_per_cta;
-  const int grid = lm_head_grid(vocab, &tiles_per_cta);
+  int rows_per_cta;
+  const int grid = lm_head_grid(vocab, &rows_per_cta);
   if (launch_lm_head(tm_w, tm_h, 0, B, bp, d_model, vocab, verdict_ids, n_verdict, part_max, part_sum, vlog, nullptr,
                      status, s) != cudaSuccess ||
       launch_gate(part_max, part_sum, grid, bp, vlog, n_verdict, B, tau, out_conf, out_accept, out_verdict, out_lse,
