@@ -34,7 +34,8 @@ enum {
   CS_ECUDA = 3,    /* a CUDA runtime / driver call failed; see cs_last_cuda_error */
   CS_ETIMEOUT = 4, /* a kernel gave up on a bounded wait (reported by cs_last_status) */
   CS_ESTATE = 5,   /* the call does not fit the handle's state (e.g. sequence not set) */
-  CS_ELIMIT = 6    /* a size exceeds the fixed capacity of an entry point that never allocates */
+  CS_ELIMIT = 6,   /* a size exceeds the fixed capacity of an entry point that never allocates */
+  CS_ERANGE = 7    /* a device-side range check of a debug build failed, or a workspace's guard bytes were written */
 };
 
 typedef struct cs_model cs_model;
@@ -336,6 +337,20 @@ int cs_last_status(cs_model* model, void* stream);
  * cs_last_status returns CS_ETIMEOUT and clears it), CS_ESTATE if the wait returned as satisfied. Synchronises `stream`.
  */
 int cs_selftest_wait_timeout(cs_model* model, int polls, void* stream);
+/*
+ * Debugging aids (there is no memory checker to run the kernels under).
+ *  - A library compiled with -DCS_DEBUG (cs_debug_build() returns 1) tests page ids, token rows and tensor-memory
+ *    columns on the device where they are used. A failed test raises a bit of the model's status word, the access is
+ *    skipped or clamped, nothing traps; the next cs_last_status returns CS_ERANGE once. The release build has none of
+ *    these tests (the host validates every argument before a launch).
+ *  - cs_selftest_range_check launches a kernel whose one range test fails by construction without touching memory:
+ *    afterwards cs_last_status returns CS_ERANGE in a debug build and CS_OK in a release build.
+ *  - Every workspace of a model (activations, staging, partial results) is followed by 256 guard bytes of a fixed
+ *    pattern. cs_check_workspace reads them back (synchronising `stream`): CS_ERANGE if any was written, in any build.
+ */
+int cs_debug_build(void);
+int cs_selftest_range_check(cs_model* model, void* stream);
+int cs_check_workspace(cs_model* model, void* stream);
 
 /*
  * Per-stage entry points. They run single kernels of the pass on caller-provided device buffers so that

@@ -11,14 +11,14 @@ import numpy as np
 
 from . import build as _build
 
-CS_OK, CS_EINVAL, CS_ENOMEM, CS_ECUDA, CS_ETIMEOUT, CS_ESTATE, CS_ELIMIT = range(7)
+CS_OK, CS_EINVAL, CS_ENOMEM, CS_ECUDA, CS_ETIMEOUT, CS_ESTATE, CS_ELIMIT, CS_ERANGE = range(8)
 
 EXPORTED = [
     "cs_version", "cs_strerror", "cs_last_cuda_error", "cs_model_load", "cs_model_free", "cs_model_set_lm_head_rows",
     "cs_reserve",
     "cs_kv_alloc", "cs_kv_alloc_8bit", "cs_kv_free", "cs_kv_pool_bytes", "cs_kv_set_seq", "cs_kv_fill", "cs_prefill",
     "cs_verify_steps", "cs_verify_cascade", "cs_append_accepted", "cs_escalate_mask", "cs_cascade_select", "cs_set_keep_logits", "cs_set_deterministic", "cs_get_last_logits", "cs_get_last_lse",
-    "cs_last_status", "cs_selftest_wait_timeout", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
+    "cs_last_status", "cs_selftest_wait_timeout", "cs_debug_build", "cs_selftest_range_check", "cs_check_workspace", "cs_gemm_f16", "cs_rmsnorm", "cs_lm_head_gate", "cs_lm_head_gate_static", "cs_take_launch_count", "cs_last_h2d_bytes", "cs_profile", "cs_profile_read",
 ]
 
 PROF_CLASSES = ["embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gateup", "gemm_down",
@@ -87,6 +87,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "cs_get_last_lse": (C.c_int, [vp, vp, i32, vp]),
         "cs_last_status": (C.c_int, [vp, vp]),
         "cs_selftest_wait_timeout": (C.c_int, [vp, i32, vp]),
+        "cs_debug_build": (C.c_int, []),
+        "cs_selftest_range_check": (C.c_int, [vp, vp]),
+        "cs_check_workspace": (C.c_int, [vp, vp]),
         "cs_gemm_f16": (C.c_int, [vp, vp, vp, vp, i32, i32, i32, i32, vp]),
         "cs_rmsnorm": (C.c_int, [vp, vp, vp, i32, i32, f32, vp]),
         "cs_lm_head_gate": (C.c_int, [vp, vp, i32, i32, i32, vp, i32, f32, vp, vp, vp, vp, vp]),
@@ -345,6 +348,18 @@ def cs_last_status(model: int, stream=None) -> None:
 
 def cs_selftest_wait_timeout(model: int, polls: int = 4096, stream=None) -> None:
     _check(load_library().cs_selftest_wait_timeout(model, int(polls), _stream_ptr(stream)), "cs_selftest_wait_timeout")
+
+
+def cs_debug_build() -> bool:
+    return bool(load_library().cs_debug_build())
+
+
+def cs_selftest_range_check(model: int, stream=None) -> None:
+    _check(load_library().cs_selftest_range_check(model, _stream_ptr(stream)), "cs_selftest_range_check")
+
+
+def cs_check_workspace(model: int, stream=None) -> None:
+    _check(load_library().cs_check_workspace(model, _stream_ptr(stream)), "cs_check_workspace")
 
 
 def cs_gemm_f16(a, w, w2, out, M: int, N: int, K: int, epilogue: int, stream=None) -> None:

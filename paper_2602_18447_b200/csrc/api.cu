@@ -39,6 +39,11 @@ struct LayerDev {
   CUtensorMap tm_wqkv, tm_wo, tm_wg, tm_wu, tm_wd;
 };
 
+// A workspace buffer. Behind its `cap` usable bytes lie kCanaryBytes of a fixed pattern that nothing may write: a
+// kernel that runs past the end of a workspace disturbs them, which cs_check_workspace finds.
+constexpr size_t kCanaryBytes = 256;
+constexpr int kCanaryByte = 0xC5;
+
 struct DevBuf {
   void* p = nullptr;
   size_t cap = 0;
@@ -50,12 +55,25 @@ struct DevBuf {
       p = nullptr;
       cap = 0;
     }
-    const size_t want = bytes + bytes / 4 + 256;
-    cudaError_t e = cudaMalloc(&p, want);
+    const size_t want = ((bytes + bytes / 4 + 256) + 255) & ~static_cast<size_t>(255);
+    cudaError_t e = cudaMalloc(&p, want + kCanaryBytes);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(workspace)");
     if (zero && (e = cudaMemset(p, 0, want)) != cudaSuccess) return cuda_fail(e, "cudaMemset(workspace)");
+    if ((e = cudaMemset(static_cast<uint8_t*>(p) + want, kCanaryByte, kCanaryBytes)) != cudaSuccess)
+      return cuda_fail(e, "cudaMemset(workspace canary)");
     cap = want;
     return CS_OK;
+  }
+  // 0 = intact, 1 = disturbed, -1 = the read-back failed
+  int canary_state(cudaStream_t s) const {
+    if (!p) return 0;
+    uint8_t h[kCanaryBytes];
+    if (cudaMemcpyAsync(h, static_cast<const uint8_t*>(p) + cap, kCanaryBytes, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+      return -1;
+    for (size_t i = 0; i < kCanaryBytes; ++i)
+      if (h[i] != kCanaryByte) return 1;
+    return 0;
   }
   void release() {
     if (p) cudaFree(p);
@@ -398,7 +416,7 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
     return CS_ECUDA;
   }
 
-  CS_STEP(kProfEmbed, launch_embed(d_tok, m->embed, x, T, d.d_model, d.vocab, s));
+  CS_STEP(kProfEmbed, launch_embed(d_tok, m->embed, x, T, d.d_model, d.vocab, m->status, s));
   CS_STEP(kProfOther, launch_rope_table(d_pos, m->inv_freq, rope, T, d.head_dim / 2, s));
 
   AttnParams ap;
@@ -415,6 +433,8 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
   ap.part_ml = static_cast<float*>(m->attn_part_ml.p);
   ap.counters = static_cast<int32_t*>(m->attn_counters.p);
   ap.status = m->status;
+  ap.num_pages = kv->num_pages;
+  ap.n_rows = T;
   const int plane_groups = kv->num_pages * d.n_kv_heads * kPageSize / 8;
 
   TurnOrder turn_order{m->turn_flags, &m->turn_epoch};
@@ -436,7 +456,7 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
                                 append_kv->table_dev, append_kv->max_pages_per_seq,
                                 append_kv->pool + static_cast<size_t>(2 * l) * append_kv->plane_elems,
                                 append_kv->pool + static_cast<size_t>(2 * l + 1) * append_kv->plane_elems,
-                                d.n_kv_heads, d.head_dim, kPageSize, T, 1, s));
+                                d.n_kv_heads, d.head_dim, kPageSize, T, 1, append_kv->num_pages, m->status, s));
       break;
     }
     if (kv->format != 0) {
@@ -452,7 +472,7 @@ int run_layers(cs_model* m, const cs_kv* kv, cs_kv* append_kv, const BatchLayout
                                 append_kv->table_dev, append_kv->max_pages_per_seq,
                                 append_kv->pool + static_cast<size_t>(2 * l) * append_kv->plane_elems,
                                 append_kv->pool + static_cast<size_t>(2 * l + 1) * append_kv->plane_elems,
-                                d.n_kv_heads, d.head_dim, kPageSize, T, 1, s));
+                                d.n_kv_heads, d.head_dim, kPageSize, T, 1, append_kv->num_pages, m->status, s));
     }
     CS_STEP(kProfO, gemm_f16(tm_o, lw.tm_wo, nullptr, x, T, d.d_model, m->q_dim, kEpiResidAdd, m->status, s, turn));
     if (l == d.n_layers - 1 && !append_kv) {
@@ -603,6 +623,7 @@ const char* cs_strerror(int status) {
     case CS_ETIMEOUT: return "a kernel gave up on a bounded wait";
     case CS_ESTATE: return "call does not fit the handle's state";
     case CS_ELIMIT: return "size exceeds the fixed capacity of an entry point that never allocates";
+    case CS_ERANGE: return "a range check failed: an index left its array (debug build) or a workspace's guard bytes were written";
     default: return "unknown status";
   }
 }
@@ -911,7 +932,7 @@ int cs_kv_fill(cs_kv* kv, int seq, int layer, const uint16_t* host_k, const uint
   CS_CUDA(launch_kv_scatter(tk, tv, static_cast<int>(row), nullptr, nullptr, seq, 0, kv->table_dev,
                             kv->max_pages_per_seq, kv->pool + static_cast<size_t>(2 * layer) * kv->plane_elems,
                             kv->pool + static_cast<size_t>(2 * layer + 1) * kv->plane_elems, d.n_kv_heads, d.head_dim,
-                            kPageSize, c, 0, s));
+                            kPageSize, c, 0, kv->num_pages, nullptr, s));
   CS_CUDA(cudaStreamSynchronize(s));
   return CS_OK;
 }
@@ -1185,7 +1206,35 @@ int cs_last_status(cs_model* m, void* stream) {
   CS_CUDA(cudaMemcpyAsync(&v, m->status, 4, cudaMemcpyDeviceToHost, s));
   CS_CUDA(cudaStreamSynchronize(s));
   if (v) CS_CUDA(cudaMemsetAsync(m->status, 0, 4, s));
-  return (v & 1u) ? CS_ETIMEOUT : CS_OK;
+  return (v & 1u) ? CS_ETIMEOUT : (v & 2u) ? CS_ERANGE : CS_OK;
+}
+
+int cs_check_workspace(cs_model* m, void* stream) {
+  if (!m) return CS_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const DevBuf* bufs[] = {&m->x, &m->x_last, &m->a, &m->qkv, &m->attn_o, &m->hmlp, &m->rope, &m->h_last, &m->lm_part,
+                          &m->vlogits, &m->logits, &m->lse, &m->attn_part_o, &m->attn_part_ml, &m->attn_counters,
+                          &m->stg.dev, &m->casc_idx, &m->casc_conf, &m->casc_verdict, &m->casc_accept};
+  for (const DevBuf* b : bufs) {
+    const int st = b->canary_state(s);
+    if (st < 0) return cuda_fail(cudaGetLastError(), "workspace canary read-back");
+    if (st > 0) return CS_ERANGE;
+  }
+  return CS_OK;
+}
+
+int cs_selftest_range_check(cs_model* m, void* stream) {
+  if (!m) return CS_EINVAL;
+  CS_CUDA(launch_range_check_selftest(m->status, static_cast<cudaStream_t>(stream)));
+  return CS_OK;
+}
+
+int cs_debug_build(void) {
+#ifdef CS_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
 }
 
 int cs_selftest_wait_timeout(cs_model* m, int polls, void* stream) {

@@ -346,8 +346,18 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_pool
     // Lane l < 8 fetches page l of a cached tile. Pages past the end of the context are replaced by the last
     // real page; their keys are masked.
     auto page_of = [&](int t) -> int {
-      return (t < ctx_tiles && lane < kPagesPerTile) ? __ldg(pages + min(t * kPagesPerTile + lane, n_pages - 1)) : 0;
+      if (!(t < ctx_tiles && lane < kPagesPerTile)) return 0;
+      const int id = __ldg(pages + min(t * kPagesPerTile + lane, n_pages - 1));
+      return debug_in_range(id >= 0 && id < p.num_pages, p.status) ? id : 0;
     };
+    // token rows of this item lie inside the batch, its key tiles inside its sequence, its tensor-memory buffers
+    // inside the allocation
+    if (lane == 0) {
+      debug_in_range(tok0 >= 0 && n_new > 0 && tok0 + n_new <= p.n_rows && it.q_tok0 >= 0 && it.q_tok0 < n_new, p.status);
+      debug_in_range(it.tile_begin >= 0 && it.tile_begin < it.tile_end &&
+                     it.tile_end <= ctx_tiles + (n_new + kKTile - 1) / kKTile && n_pages <= p.max_pages_per_seq, p.status);
+      debug_in_range(L::kOCol + HD <= L::kTmemCols && kSBufs * kKTile <= static_cast<int>(L::kOCol), p.status);
+    }
     int page = page_of(it.tile_begin);
     // column of this kv head's K (or V) in the qkv workspace, in 64-column units
     const int col = (p.n_q_heads + (is_k ? 0 : p.n_kv_heads) + it.kv_head) * L::kHalves;

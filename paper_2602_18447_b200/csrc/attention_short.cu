@@ -123,6 +123,7 @@ attention_short_kernel(const AttnParams p, const uint8_t* __restrict__ pool_k, c
   // cached pages of this warp: page_begin + warp, + 4, ...; the copies touch only the cache and the page table, which
   // no kernel of the pass writes, so the first ones go out before the wait on the previous kernel
   auto fetch = [&](int32_t id, int stage) {
+    if (!debug_in_range(id >= 0 && id < p.num_pages, p.status)) id = 0;
     const uint8_t* gk = pool_k + static_cast<size_t>(id) * page_stride + head_off;
     const uint8_t* gv = pool_v + static_cast<size_t>(id) * page_stride + head_off;
     uint8_t* dst = my + stage * STAGE;

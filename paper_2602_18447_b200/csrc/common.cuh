@@ -9,8 +9,25 @@
 
 namespace cs {
 
-// Status word written by kernels; bit 0 = a bounded wait ran out.
+// Status word written by kernels; bit 0 = a bounded wait ran out, bit 1 = a range check of a debug build failed.
 constexpr uint32_t kStatusTimeout = 1u;
+constexpr uint32_t kStatusRange = 2u;
+
+// Range checks of a build with -DCS_DEBUG: page ids, token rows and tensor-memory columns are tested where they are
+// used. A failed check raises bit 1 of the status word (cs_last_status then returns CS_ERANGE) and tells the caller
+// to skip or clamp the access; it never traps, so the context stays usable. Without CS_DEBUG the checks compile away.
+#ifdef CS_DEBUG
+constexpr bool kDebugChecks = true;
+#else
+constexpr bool kDebugChecks = false;
+#endif
+__device__ __forceinline__ bool debug_in_range(bool in_range, uint32_t* status) {
+  if (kDebugChecks && !in_range) {
+    atomicOr(status, kStatusRange);
+    return false;
+  }
+  return true;
+}
 
 // Upper bound on polls of one mbarrier wait. Each poll is a try_wait that may itself suspend for a short
 // hardware-defined time, so the bound is reached after seconds at most, never in a healthy run.

@@ -11,11 +11,12 @@ namespace {
 thread_local int64_t g_launches = 0;
 
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const uint16_t* __restrict__ embed,
-                             float* __restrict__ x, int T, int d, int vocab) {
+                             float* __restrict__ x, int T, int d, int vocab, uint32_t* status) {
   pdl_launch_dependents();
   pdl_wait();
   const int t = blockIdx.x;
   int tok = tokens[t];
+  if (threadIdx.x == 0) debug_in_range(tok >= 0 && tok < vocab, status);
   tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);
   const uint4* src = reinterpret_cast<const uint4*>(embed + static_cast<size_t>(tok) * d);
   float4* dst = reinterpret_cast<float4*>(x + static_cast<size_t>(t) * d);
@@ -105,7 +106,8 @@ __global__ void kv_scatter_kernel(const uint16_t* __restrict__ src_k, const uint
                                   const int32_t* __restrict__ tok_pos, int const_seq, int pos0,
                                   const int32_t* __restrict__ page_table,
                                   int max_pages_per_seq, uint16_t* __restrict__ pool_k, uint16_t* __restrict__ pool_v,
-                                  int n_kv_heads, int hd, int page_size, int T, int src_is_f16) {
+                                  int n_kv_heads, int hd, int page_size, int T, int src_is_f16, int num_pages,
+                                  uint32_t* status) {
   pdl_launch_dependents();
   pdl_wait();
   const int chunks = n_kv_heads * hd / 8;
@@ -117,7 +119,9 @@ __global__ void kv_scatter_kernel(const uint16_t* __restrict__ src_k, const uint
   const int e = c * 8 - head * hd;
   const int pos = tok_seq ? tok_pos[t] : pos0 + t;
   const int seq = tok_seq ? tok_seq[t] : const_seq;
+  if (!debug_in_range(pos >= 0 && pos / page_size < max_pages_per_seq, status)) return;
   const int page = page_table[static_cast<size_t>(seq) * max_pages_per_seq + pos / page_size];
+  if (!debug_in_range(page >= 0 && page < num_pages, status)) return;
   const int slot = pos % page_size;
   const size_t dst = ((static_cast<size_t>(page) * n_kv_heads + head) * page_size + slot) * hd + e;
   const size_t src = static_cast<size_t>(t) * row_stride + c * 8;
@@ -180,7 +184,18 @@ __global__ void wait_timeout_selftest_kernel(uint32_t* status, uint32_t limit, i
   }
 }
 
+__global__ void range_check_selftest_kernel(uint32_t* status) {
+  const int index = 7, extent = 4;                  // out of range by construction; nothing is accessed
+  debug_in_range(index < extent, status);
+}
+
 }  // namespace
+
+cudaError_t launch_range_check_selftest(uint32_t* status, cudaStream_t s) {
+  range_check_selftest_kernel<<<1, 1, 0, s>>>(status);
+  count_launch();
+  return cudaGetLastError();
+}
 
 cudaError_t launch_wait_timeout_selftest(uint32_t* status, uint32_t limit, int32_t* gave_up, cudaStream_t s) {
   wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status, limit, gave_up);
@@ -202,9 +217,9 @@ int64_t take_launch_count() {
 }
 
 cudaError_t launch_embed(const int32_t* tokens, const uint16_t* embed, float* x, int T, int d, int vocab,
-                         cudaStream_t s) {
+                         uint32_t* status, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
-  cudaError_t le = launch_pdl(embed_kernel, dim3(T), dim3(128), 0, s, tokens, embed, x, T, d, vocab);
+  cudaError_t le = launch_pdl(embed_kernel, dim3(T), dim3(128), 0, s, tokens, embed, x, T, d, vocab, status);
   count_launch();
   return le != cudaSuccess ? le : cudaGetLastError();
 }
@@ -235,12 +250,12 @@ cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int 
                               const int32_t* tok_pos, int const_seq, int pos0, const int32_t* page_table,
                               int max_pages_per_seq,
                               uint16_t* pool_k_plane, uint16_t* pool_v_plane, int n_kv_heads, int hd, int page_size,
-                              int T, int src_is_f16, cudaStream_t s) {
+                              int T, int src_is_f16, int num_pages, uint32_t* status, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   const int n = T * n_kv_heads * hd / 8;
   kv_scatter_kernel<<<(n + 255) / 256, 256, 0, s>>>(src_k, src_v, row_stride, tok_seq, tok_pos, const_seq, pos0, page_table,
                                                     max_pages_per_seq, pool_k_plane, pool_v_plane, n_kv_heads, hd,
-                                                    page_size, T, src_is_f16);
+                                                    page_size, T, src_is_f16, num_pages, status);
   count_launch();
   return cudaGetLastError();
 }

@@ -360,6 +360,8 @@ gemm_f16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, status)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
+      // the tile lies inside the output and its accumulator inside the tensor-memory allocation
+      if (lane == 0) debug_in_range(m0 >= 0 && m0 < M && n0 >= 0 && n0 < N && acc * BN + BN <= static_cast<int>(kTmemCols), status);
       uint32_t r[32];
       if (EPI == kEpiSwiGLU) {
         uint32_t r2[32];

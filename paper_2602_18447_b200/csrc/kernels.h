@@ -59,10 +59,12 @@ struct AttnParams {
   float* part_ml;           // [slots, 128, 2]  exponent reference (raw score units) and sum
   int32_t* counters;        // [slots] zero between launches
   uint32_t* status;
+  int32_t num_pages;        // pages of the pool and rows of the qkv workspace in use: range checks of debug builds
+  int32_t n_rows;
 };
 
 cudaError_t launch_embed(const int32_t* tokens, const uint16_t* embed, float* x, int T, int d, int vocab,
-                         cudaStream_t s);
+                         uint32_t* status, cudaStream_t s);
 cudaError_t launch_rmsnorm(const float* x, const float* gain, uint16_t* out, int rows, int d, float eps,
                            cudaStream_t s);
 // cos/sin of pos[t] * inv_freq[j] in double, stored as float2 [T, half].
@@ -76,7 +78,7 @@ cudaError_t launch_kv_scatter(const uint16_t* src_k, const uint16_t* src_v, int 
                               const int32_t* tok_pos, int const_seq, int pos0, const int32_t* page_table,
                               int max_pages_per_seq,
                               uint16_t* pool_k_plane, uint16_t* pool_v_plane, int n_kv_heads, int hd, int page_size,
-                              int T, int src_is_f16, cudaStream_t s);
+                              int T, int src_is_f16, int num_pages, uint32_t* status, cudaStream_t s);
 // Re-encode n bf16 values (n even) as fp16 in place.
 cudaError_t launch_bf16_to_f16(uint16_t* p, size_t n, cudaStream_t s);
 
@@ -132,6 +134,10 @@ cudaError_t launch_cascade_scatter(int B, const uint8_t* trusted, const int32_t*
                                    const int32_t* idx, const int32_t* count, const int32_t* verdict_c,
                                    const float* conf_c, int32_t* out_verdict_t, float* out_conf_t,
                                    int32_t* out_verdict, float* out_conf, cudaStream_t s);
+
+// Evaluates one range check that fails by construction (no memory is touched): in a debug build the status word gets
+// its range bit, in a release build nothing happens.
+cudaError_t launch_range_check_selftest(uint32_t* status, cudaStream_t s);
 
 // Failure-detection self-test: a bounded wait that is made to run out (see cs_selftest_wait_timeout).
 cudaError_t launch_wait_timeout_selftest(uint32_t* status, uint32_t limit, int32_t* gave_up, cudaStream_t s);

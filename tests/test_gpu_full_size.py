@@ -51,6 +51,7 @@ def _run_full(name, weights, n_sample, always=()):
         vid = list(cfg.verdict_ids)
         assert np.max(np.abs(np.exp(z[:, vid] - lse_from_logits[:, None]).max(axis=1) - gpu["conf"])) < 1e-6
         del z
+        B.cs_check_workspace(ses.model)          # guard bytes behind every workspace are intact
         # the pass is deterministic: a second run gives the same bits (logits of all steps, confidences, mask)
         ses.verify()
         again = ses.results()

@@ -43,6 +43,9 @@ def _run(cfg, weights, batch, taus=None, planted=False, both_sides=False):
                 P.compare(g2, None, r2, tau)
         if both_sides:
             assert n_tr >= 1 and n_es >= 1, (n_tr, n_es, ref["conf"])
+        # nothing wrote past the end of a workspace (guard bytes behind every buffer)
+        from paper_2602_18447_b200 import binding as B
+        B.cs_check_workspace(ses.model)
         # host-token entry (tokens copied inside the call): the same pass, bit for bit (every reduction of the pass has
         # a fixed order), logits included
         ses.verify(host_tokens=True)
