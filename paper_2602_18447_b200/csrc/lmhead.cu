@@ -23,8 +23,9 @@ constexpr int kLmMaxVerdict = 8;
 template <int NB>
 struct LmSmem {
   static constexpr int kHBytes = NB * kLmBK * 2;
-  static constexpr int kStageBytes = kLmWBytes + ((kHBytes + 1023) / 1024) * 1024;
-  static constexpr int kStages = 8;
+  // a stage: two 128-row tiles of W (a 256-row "double tile") and the one tile of hidden states they share
+  static constexpr int kStageBytes = 2 * kLmWBytes + ((kHBytes + 1023) / 1024) * 1024;
+  static constexpr int kStages = 5;
   static constexpr int kBarOff = kStages * kStageBytes;
   static constexpr int kRedOff = kBarOff + 256;                 // [4 warps][NB][2] floats
   static constexpr int kTotal = kRedOff + 4 * NB * 2 * 4 + 1024;
@@ -68,9 +69,42 @@ __device__ __forceinline__ bool lm_kblock_peek(uint32_t tmem_d, uint64_t adesc, 
   return ready != 0;
 }
 
+// The same for a double tile: the second 128 rows of W lie 16 KB behind the first in the stage and accumulate NB
+// columns further on in tensor memory; both read the same hidden-state tile.
+__device__ __forceinline__ bool lm_kblock2_peek(uint32_t tmem_d, uint32_t tmem_d2, uint64_t adesc, uint64_t bdesc,
+                                                uint32_t idesc, uint32_t accumulate_first, uint64_t* commit_bar,
+                                                uint64_t* peek_bar, uint32_t peek_parity) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred P, Q;\n\t.reg .b64 a1, a2, a3, b1, b2, b3, c0, c1, c2, c3;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "setp.ne.b32 Q, %7, 0;\n\t"
+      "add.u64 a1, %4, 2;\n\tadd.u64 b1, %5, 2;\n\t"
+      "add.u64 a2, %4, 4;\n\tadd.u64 b2, %5, 4;\n\t"
+      "add.u64 a3, %4, 6;\n\tadd.u64 b3, %5, 6;\n\t"
+      "add.u64 c0, %4, 1024;\n\tadd.u64 c1, %4, 1026;\n\tadd.u64 c2, %4, 1028;\n\tadd.u64 c3, %4, 1030;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, Q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%9], c0, %5, %6, Q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], a1, b1, %6, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%9], c1, b1, %6, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], a2, b2, %6, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%9], c2, b2, %6, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%3], a3, b3, %6, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%9], c3, b3, %6, 1;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ready)
+      : "r"(smem_u32(peek_bar)), "r"(peek_parity), "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc),
+        "r"(accumulate_first), "r"(smem_u32(commit_bar)), "r"(tmem_d2)
+      : "memory");
+  return ready != 0;
+}
+
 // Rows of the vocabulary [blockIdx.x * rows_per_cta, + rows_per_cta) belong to a CTA, cut evenly so that every SM
-// streams the same number of bytes. A range is walked in 128-row tiles; when it is not a multiple of 128 its last,
-// partial tile comes FIRST: the rows that tile fetches beyond the range are the first tile of the next CTA, which
+// streams the same number of bytes. A range is walked in 256-row double tiles (two products per tile of hidden states:
+// with 32-64 steps per pass the hidden states re-read from L2 for every tile of W are half as many bytes again as W
+// itself, more than an SM takes in at the clock the power cap leaves); when the range is not a multiple of 256 its
+// last, partial double tile (one 128-row tile if that covers it) comes FIRST: the rows that tile fetches beyond the range are the first tile of the next CTA, which
 // fetches them at the same moment, so they cross the DRAM interface once.
 struct LmArgs {
   int B, vocab, kblocks, rows_per_cta, n_verdict, h_row0;
@@ -86,7 +120,7 @@ template <int NB>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const LmArgs a) {
   using L = LmSmem<NB>;
-  constexpr uint32_t kTmemCols = (2 * NB < 32) ? 32 : 2 * NB;
+  constexpr uint32_t kTmemCols = (4 * NB < 32) ? 32 : 4 * NB;     // two accumulators of two tiles of NB columns
   constexpr uint32_t kIdesc = umma_idesc_f16(kLmBM, NB);
 
   extern __shared__ uint8_t smem_raw[];
@@ -103,13 +137,15 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row_begin = blockIdx.x * a.rows_per_cta;
   const int row_end = min(a.vocab, row_begin + a.rows_per_cta);
-  const int n_my_tiles = (row_end - row_begin + kLmBM - 1) / kLmBM;
-  const bool tail_first = ((row_end - row_begin) % kLmBM) != 0 && n_my_tiles > 1;
-  // first row of the i-th tile this CTA works on
+  constexpr int kDouble = 2 * kLmBM;
+  const int n_my_tiles = (row_end - row_begin + kDouble - 1) / kDouble;
+  const bool tail_first = ((row_end - row_begin) % kDouble) != 0 && n_my_tiles > 1;
+  // first row of the i-th double tile this CTA works on, and whether its second 128 rows hold any row of the range
   auto tile_row0 = [&](int i) {
     const int t = tail_first ? (i == 0 ? n_my_tiles - 1 : i - 1) : i;
-    return row_begin + t * kLmBM;
+    return row_begin + t * kDouble;
   };
+  auto tile_is_double = [&](int i) { return tile_row0(i) + kLmBM < row_end; };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < L::kStages; ++s) {
@@ -143,12 +179,14 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
       bool ok = true;
       for (int i = 0; i < n_my_tiles && ok; ++i) {
         const int r0 = tile_row0(i);
+        const bool two = tile_is_double(i);
         for (int kb = 0; kb < a.kblocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, a.status)) { ok = false; break; }
           uint8_t* sw = smem + stage * L::kStageBytes;
-          mbar_arrive_expect_tx(&full_bar[stage], kLmWBytes + L::kHBytes);
+          mbar_arrive_expect_tx(&full_bar[stage], (two ? 2 : 1) * kLmWBytes + L::kHBytes);
           tma_load_2d(sw, &tm_w, &full_bar[stage], kb * kLmBK, r0);
-          tma_load_2d(sw + kLmWBytes, &tm_h, &full_bar[stage], kb * kLmBK, a.h_row0);
+          if (two) tma_load_2d(sw + kLmWBytes, &tm_w, &full_bar[stage], kb * kLmBK, r0 + kLmBM);
+          tma_load_2d(sw + 2 * kLmWBytes, &tm_h, &full_bar[stage], kb * kLmBK, a.h_row0);
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -162,17 +200,20 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
       bool ok = true, ready = false;
       const uint32_t smem_base = smem_u32(smem);
       const uint64_t adesc0 = umma_desc_k128(smem_base);
-      const uint64_t bdesc0 = umma_desc_k128(smem_base + kLmWBytes);
+      const uint64_t bdesc0 = umma_desc_k128(smem_base + 2 * kLmWBytes);
       for (int i = 0; i < n_my_tiles && ok; ++i) {
         if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * NB;
+        const uint32_t d_tmem = tmem_base + acc * 2 * NB;
+        const bool two = tile_is_double(i);
         for (int kb = 0; kb < a.kblocks; ++kb) {
           if (!ready && !mbar_wait(&full_bar[stage], phase, abort_flag, a.status)) { ok = false; break; }
           const int ns = (stage + 1 == L::kStages) ? 0 : stage + 1;
           const uint32_t np = (ns == 0) ? phase ^ 1u : phase;
           const uint64_t off = static_cast<uint64_t>(stage * (L::kStageBytes >> 4));
-          ready = lm_kblock_peek(d_tmem, adesc0 + off, bdesc0 + off, kIdesc, kb != 0, &empty_bar[stage], &full_bar[ns], np);
+          ready = two ? lm_kblock2_peek(d_tmem, d_tmem + NB, adesc0 + off, bdesc0 + off, kIdesc, kb != 0, &empty_bar[stage],
+                                        &full_bar[ns], np)
+                      : lm_kblock_peek(d_tmem, adesc0 + off, bdesc0 + off, kIdesc, kb != 0, &empty_bar[stage], &full_bar[ns], np);
           stage = ns;
           phase = np;
         }
@@ -193,8 +234,11 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     for (int i = 0; i < n_my_tiles; ++i) {
       if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, a.status)) { ok = false; break; }
       tc_fence_after();
-      const uint32_t t_row = tmem_base + acc * NB + (static_cast<uint32_t>(quad * 32) << 16);
-      const int row = tile_row0(i) + quad * 32 + lane;   // vocabulary id of this thread's lane
+      const int n_sub = tile_is_double(i) ? 2 : 1;
+#pragma unroll 1
+      for (int sub = 0; sub < n_sub; ++sub) {
+      const uint32_t t_row = tmem_base + acc * 2 * NB + sub * NB + (static_cast<uint32_t>(quad * 32) << 16);
+      const int row = tile_row0(i) + sub * kLmBM + quad * 32 + lane;   // vocabulary id of this thread's lane
       const bool row_ok = row < row_end;                 // rows past the range belong to the next CTA (or to nobody)
       uint32_t vmask = 0;   // which entries of verdict_ids name this row (an id may be listed twice)
       for (int j = 0; j < a.n_verdict; ++j)
@@ -218,6 +262,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             }
           }
         }
+      }
       }
       tc_fence_before();
       __syncwarp();
