@@ -199,3 +199,32 @@ def test_without_the_fixed_order_passes_agree_to_rounding():
         P.compare_planted(b, ses.last_logits(), ref, cfg.tau, cfg, gpu_lse=ses.last_lse())
     finally:
         ses.close()
+
+
+def test_splitting_the_batch_changes_nothing_beyond_rounding():
+    """Steps are verified independently (Section 4.3): one call over the batch and two calls over its halves give the
+    same confidences up to the rounding order of the residual projections (whose pieces depend on the token count)."""
+    import torch
+    from paper_2602_18447_b200 import binding as B
+    cfg = replace(get_config("cfg1_tiny"), batch=10, ctx_dist=("uniform", 20, 150), step_dist=("uniform", 5, 60))
+    w, batch = P.planted_weights(cfg), make_batch(cfg)
+    ses = P.build_session(cfg, w, batch)
+    try:
+        ses.verify()
+        whole = ses.results()
+        parts = []
+        for lo, hi in ((0, 4), (4, 10)):
+            toks = np.concatenate(P.steps_of(batch)[lo:hi]).astype(np.int32)
+            conf = torch.empty(hi - lo, dtype=torch.float32, device="cuda")
+            acc = torch.empty(hi - lo, dtype=torch.uint8, device="cuda")
+            B.cs_verify_steps(ses.model, ses.kv, np.arange(lo, hi, dtype=np.int32), toks, batch.step_lens[lo:hi],
+                              cfg.verdict_ids, cfg.tau, conf, acc)
+            torch.cuda.synchronize()
+            parts.append((conf.cpu().numpy(), acc.cpu().numpy()))
+        conf2 = np.concatenate([p[0] for p in parts])
+        acc2 = np.concatenate([p[1] for p in parts])
+        assert np.max(np.abs(conf2 - whole["conf"])) <= 2.5e-3
+        sure = np.abs(whole["conf"] - cfg.tau) > 2.5e-3
+        assert np.array_equal(acc2[sure], whole["accept"][sure])
+    finally:
+        ses.close()
