@@ -601,7 +601,24 @@ cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorM
     upc = tpc * kblocks;
   }
   CUtensorMap tout = ta;   // only the residual epilogue reads it
-  if (EPI == kEpiResidAdd && !make_out_f32_map(&tout, out, M, N)) return cudaErrorInvalidValue;
+  if (EPI == kEpiResidAdd) {
+    // The output of the residual projections is the same buffer and shape for every layer of a pass (x, and the last
+    // rows' copy of it): its tensor map is encoded when either changes, not per launch.
+    struct OutMap { void* base = nullptr; int rows = 0, cols = 0; CUtensorMap tm; };
+    thread_local OutMap cache[2];
+    thread_local int next = 0;
+    const OutMap* hit = nullptr;
+    for (const OutMap& c : cache)
+      if (c.base == out && c.rows == M && c.cols == N) hit = &c;
+    if (!hit) {
+      OutMap& c = cache[next];
+      next ^= 1;
+      if (!make_out_f32_map(&c.tm, out, M, N)) { c.base = nullptr; return cudaErrorInvalidValue; }
+      c.base = out; c.rows = M; c.cols = N;
+      hit = &c;
+    }
+    tout = hit->tm;
+  }
   cudaError_t le = launch_pdl(gemm_f16_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), L::kTotal, stream, ta, tb, tb2, tout, out, M,
                               N, m_tiles, n_tiles, kblocks, total, upc, rope, status, turn_flags, epoch);
   count_launch();
