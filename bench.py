@@ -467,7 +467,7 @@ def run_ours(args, cfg):
         "time_shares": shares,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        sample = list(range(min(3, batch.n_steps)))
+        sample = list(range(min(6, batch.n_steps)))         # ~15 s of CPU work at the 1.5B shape
         t = oracle_sample_run(cfg, weights, batch, sample)
         out["cpu_baseline"] = {"value": len(sample) / t, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                "sample": f"one oracle pass over steps {sample} of the {batch.n_steps}-step batch "
