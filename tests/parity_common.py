@@ -85,7 +85,7 @@ def compare(gpu: dict, gpu_logits: Optional[np.ndarray], ref: dict, tau: float, 
 # The planted rows have norm beta ~ ln V + 0.5 instead of init_std * sqrt(d), so the same direction error of the last
 # hidden state (the fp16 rounding of the activations, accumulated over the layers) moves their logits further than an
 # ordinary row's. The bounds below are not derived from that worst case: they are at most three times the largest
-# error observed on the GPU for the class of model (see the table of observed maxima in the design notes), so a
+# error observed on the GPU for the class of model (the tests record the maxima when CS_PARITY_STATS is set), so a
 # regression of the forward pass by a small factor fails them. Keys: (shallow, deep) = (up to 3 layers, more).
 # Observed worst cases: planted-row logit 2.1e-2 (shallow) / 4.8e-2 (deep), confidence 4.0e-3 / 1.1e-2.
 PLANTED_LOGIT_TOL = {"shallow": 6e-2, "deep": 1.2e-1}
