@@ -57,7 +57,8 @@ def test_gemm_matches_oracle_matmul(M, N, K, epilogue):
     assert not bad.any(), (int(bad.sum()), float(np.abs(got - want).max()), scale)
 
 
-@pytest.mark.parametrize("M,N,K", [(1163, 1536, 8960), (16, 1536, 8960), (2038, 3584, 3584), (1163, 1536, 1536), (300, 264, 4104)])
+@pytest.mark.parametrize("M,N,K", [(1163, 1536, 8960), (16, 1536, 8960), (2038, 3584, 3584), (1163, 1536, 1536), (300, 264, 4104),
+                                   (735, 1536, 8960), (64, 256, 16384), (129, 520, 2056), (1, 1536, 8960)])
 def test_residual_gemm_is_bit_identical_from_run_to_run(M, N, K):
     """Long k ranges are cut over the SMs and several CTAs add pieces into the same elements of x; with the fixed order
     of those additions ten runs on the same inputs give the same bits, also with other work on the GPU in between."""
@@ -77,6 +78,10 @@ def test_residual_gemm_is_bit_identical_from_run_to_run(M, N, K):
         runs.append(out.cpu().numpy().view(np.uint32))
     for r in runs[1:]:
         assert np.array_equal(r, runs[0])
+    # ... and it is the right sum (several pieces per tile, each added exactly once)
+    want = x0.cpu().numpy().astype(np.float64) + da.float().cpu().numpy().astype(np.float64) @ dw.float().cpu().numpy().astype(np.float64).T
+    got = runs[0].view(np.float32).astype(np.float64)
+    assert np.max(np.abs(got - want)) <= 3e-5 * float(np.abs(want).max()) * (1 + K / 1024)
 
 
 @pytest.mark.parametrize("rows,d", [(1, 256), (37, 1536), (1088, 1536), (70, 3584)])
